@@ -1,0 +1,173 @@
+/*
+ * CPU checker for the CCD compression cycle of InfiniPot (arxiv 2410.01518).
+ *
+ * TEST INFRASTRUCTURE ONLY.  Plain, slow, double precision; one loop per
+ * definition, no blocking, no fusion, no reordering.  It shares no code with
+ * the CUDA library and must never be called from it; only the tests, the smoke
+ * check and the CPU-baseline leg of the benchmark use it.
+ *
+ * What each function follows:
+ *   ora_nuc_top      Sec. 3.3.3: "first select the Top_T highest NuC scores"
+ *   ora_cap_scores   Sec. 3.3.1, Eq. 2: sum over the CaP query rows of the
+ *                    self-attention probability towards every pot key
+ *   ora_select       Sec. 3.3.3 + Appendix B "Combine NuC and CaP" / "Final
+ *                    Token Selection": NuC slots first, the remaining |C|-T
+ *                    slots by CaP score, per head
+ *   ora_gather       Appendix B "KV-cache compression": K and V rows of the
+ *                    retained slots
+ *   ora_cycle        the four steps over every (layer, stream, kv-head) unit
+ *
+ * Readings where the paper is silent (each listed in the design notes):
+ *   - every CaP row normalises over the N pot keys only (CaP keys are not in
+ *     the pot), so each softmax row sums to 1 over the context slots;
+ *   - logits are scaled by 1/sqrt(d);
+ *   - with grouped-query attention the G query heads that share a KV head are
+ *     summed like additional CaP rows (Eq. 2 is a plain sum);
+ *   - the CaP top-(|C|-T) is taken among slots not already taken by NuC, so
+ *     exactly |C| slots survive;
+ *   - ties: the lower slot index wins, in both rankings;
+ *   - survivors keep their original order (ascending slot index).
+ *
+ * Parity pins (tests/test_oracle_pins.py): row sums = 1, column-sum total =
+ * G*P, closed forms (Q = 0, equal keys, N = 1, one dominant key), slot
+ * permutation equivariance, P=G=1 against an independent library softmax,
+ * brute-force subset enumeration for the selection on tiny pots, NuC-only and
+ * CaP-only special cases, byte-wise gather identities.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+/* ---- ranking helper: indices sorted by (value descending, index ascending) ---- */
+typedef struct { double v; int j; } ora_pair;
+
+static int ora_cmp_desc(const void *a, const void *b)
+{
+    const ora_pair *x = (const ora_pair *)a, *y = (const ora_pair *)b;
+    if (x->v > y->v) return -1;
+    if (x->v < y->v) return 1;
+    return (x->j > y->j) - (x->j < y->j);
+}
+
+static int ora_cmp_int(const void *a, const void *b)
+{
+    int x = *(const int *)a, y = *(const int *)b;
+    return (x > y) - (x < y);
+}
+
+/* The T slots with the largest aux value (ties: lower slot first), returned ascending. */
+void ora_nuc_top(const double *aux, int N, int T, int *out)
+{
+    ora_pair *p = (ora_pair *)malloc(sizeof(ora_pair) * (size_t)(N > 0 ? N : 1));
+    for (int j = 0; j < N; ++j) { p[j].v = aux[j]; p[j].j = j; }
+    qsort(p, (size_t)N, sizeof(ora_pair), ora_cmp_desc);
+    for (int r = 0; r < T; ++r) out[r] = p[r].j;
+    qsort(out, (size_t)T, sizeof(int), ora_cmp_int);
+    free(p);
+}
+
+/*
+ * Eq. 2 for one KV head.  Q holds the M = G*P query rows that attend to this
+ * head's keys ([M][d]); K holds the N pot keys ([N][d]).  For every row:
+ * s_j = q.k_j / sqrt(d), p_j = exp(s_j - max) / sum, and u_j += p_j.
+ * If row_sums is not NULL it receives sum_j p_j of every row (should be 1).
+ */
+void ora_cap_scores(const double *Q, const double *K, int M, int N, int d,
+                    double *u, double *row_sums)
+{
+    double *s = (double *)malloc(sizeof(double) * (size_t)(N > 0 ? N : 1));
+    const double scale = 1.0 / sqrt((double)d);
+    for (int j = 0; j < N; ++j) u[j] = 0.0;
+    for (int i = 0; i < M; ++i) {
+        const double *q = Q + (size_t)i * d;
+        double m = -INFINITY;
+        for (int j = 0; j < N; ++j) {
+            const double *k = K + (size_t)j * d;
+            double acc = 0.0;
+            for (int c = 0; c < d; ++c) acc += q[c] * k[c];
+            s[j] = acc * scale;
+            if (s[j] > m) m = s[j];
+        }
+        double Z = 0.0;
+        for (int j = 0; j < N; ++j) { s[j] = exp(s[j] - m); Z += s[j]; }
+        double rs = 0.0;
+        for (int j = 0; j < N; ++j) { double p = s[j] / Z; u[j] += p; rs += p; }
+        if (row_sums) row_sums[i] = rs;
+    }
+    free(s);
+}
+
+/*
+ * Per-head selection.  nuc[0..T) are the NuC slots of the stream (they are kept
+ * in every head); of the other slots the R = keep - T with the largest u are
+ * kept (ties: lower slot first).  idx[0..keep) is returned ascending.
+ */
+void ora_select(const double *u, int N, const int *nuc, int T, int keep, int *idx)
+{
+    char *taken = (char *)calloc((size_t)(N > 0 ? N : 1), 1);
+    ora_pair *p = (ora_pair *)malloc(sizeof(ora_pair) * (size_t)(N > 0 ? N : 1));
+    int n = 0, c = 0;
+    for (int r = 0; r < T; ++r) { taken[nuc[r]] = 1; idx[c++] = nuc[r]; }
+    for (int j = 0; j < N; ++j) if (!taken[j]) { p[n].v = u[j]; p[n].j = j; ++n; }
+    qsort(p, (size_t)n, sizeof(ora_pair), ora_cmp_desc);
+    for (int r = 0; r < keep - T; ++r) idx[c++] = p[r].j;
+    qsort(idx, (size_t)keep, sizeof(int), ora_cmp_int);
+    free(p);
+    free(taken);
+}
+
+/* out[r] = rows[idx[r]], byte-wise. */
+void ora_gather(const uint8_t *rows, size_t row_bytes, const int *idx, int keep, uint8_t *out)
+{
+    for (int r = 0; r < keep; ++r)
+        memcpy(out + (size_t)r * row_bytes, rows + (size_t)idx[r] * row_bytes, row_bytes);
+}
+
+/*
+ * One whole cycle over n_units independent (layer, stream, kv-head) units.
+ *   Qd   [n_units][M][d] double   the M = G*P query rows of the unit's KV head
+ *                                 (the G query heads h with h / G == kv-head,
+ *                                 P CaP rows each)
+ *   Kd   [n_units][N][d] double   the unit's pot keys
+ *   Kb,Vb[n_units][N][row_bytes]  raw storage bytes of the unit's pot rows
+ *   aux  [B][N] double            per-slot novelty, shared by all heads and
+ *                                 layers of a stream
+ *   stream_of[n_units]            which stream (row of aux) each unit belongs to
+ * Outputs:
+ *   u_out [n_units][N], idx_out [n_units][keep],
+ *   Kout, Vout [n_units][keep][row_bytes]  (may be NULL)
+ * Units are independent; with OpenMP one thread takes one unit at a time.
+ */
+void ora_cycle(const double *Qd, const double *Kd, const uint8_t *Kb, const uint8_t *Vb,
+               const double *aux, const int *stream_of, int n_units, int B, int M, int d,
+               int N, int keep, int T, size_t row_bytes,
+               double *u_out, int *idx_out, uint8_t *Kout, uint8_t *Vout)
+{
+    int *nuc = (int *)malloc(sizeof(int) * (size_t)B * (size_t)(T > 0 ? T : 1));
+    for (int b = 0; b < B; ++b) ora_nuc_top(aux + (size_t)b * N, N, T, nuc + (size_t)b * T);
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int t = 0; t < n_units; ++t) {
+        const double *Q = Qd + (size_t)t * M * d;
+        const double *K = Kd + (size_t)t * N * d;
+        double *u = u_out + (size_t)t * N;
+        int *idx = idx_out + (size_t)t * keep;
+        ora_cap_scores(Q, K, M, N, d, u, NULL);
+        ora_select(u, N, nuc + (size_t)stream_of[t] * T, T, keep, idx);
+        if (Kout) ora_gather(Kb + (size_t)t * N * row_bytes, row_bytes, idx, keep,
+                             Kout + (size_t)t * keep * row_bytes);
+        if (Vout) ora_gather(Vb + (size_t)t * N * row_bytes, row_bytes, idx, keep,
+                             Vout + (size_t)t * keep * row_bytes);
+    }
+    free(nuc);
+}
+
+/* Thread count used by ora_cycle (1 when built without OpenMP). */
+#ifdef _OPENMP
+#include <omp.h>
+void ora_set_threads(int n) { if (n > 0) omp_set_num_threads(n); }
+int ora_max_threads(void) { return omp_get_max_threads(); }
+#else
+void ora_set_threads(int n) { (void)n; }
+int ora_max_threads(void) { return 1; }
+#endif

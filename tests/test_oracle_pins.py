@@ -1,0 +1,253 @@
+"""Pins for the CPU checker: what the paper and the mathematics fix, checked
+against the checker (never the other way round)."""
+import itertools
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+
+import oracle
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def rnd(seed):
+    return np.random.default_rng(seed)
+
+
+# ---------------------------------------------------------------- Eq. 2
+def test_worked_example_eq2():
+    want = {}
+    for line in open(os.path.join(GOLD, "eq2_worked_example.txt")):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        k, v = line.split("=")
+        want[k.strip()] = float(sum(Fraction(t.strip()) for t in v.split("+")))
+    Q = np.array([[2.0, 0, 0, 0], [-2.0, 0, 0, 0]])
+    K = np.array([[0.0, 5, -1, 2], [np.log(2.0), 7, 0, 1], [np.log(3.0), -3, 4, 9]])
+    u = oracle.cap_scores(Q, K)
+    np.testing.assert_allclose(u, [want["u0"], want["u1"], want["u2"]], rtol=1e-14)
+
+
+@pytest.mark.parametrize("M,N,d", [(1, 7, 4), (16, 64, 8), (64, 512, 64), (5, 33, 128)])
+def test_rows_sum_to_one_and_total_is_M(M, N, d):
+    g = rnd(1)
+    Q, K = g.standard_normal((M, d)) * 3, g.standard_normal((N, d)) * 3
+    u, rs = oracle.cap_scores(Q, K, return_row_sums=True)
+    np.testing.assert_allclose(rs, 1.0, atol=1e-12)
+    assert abs(u.sum() - M) <= 1e-10 * M
+    assert (u >= 0).all()
+
+
+def test_zero_queries_and_equal_keys_give_uniform():
+    g = rnd(2)
+    M, N, d = 6, 40, 16
+    K = g.standard_normal((N, d))
+    np.testing.assert_allclose(oracle.cap_scores(np.zeros((M, d)), K), M / N, rtol=1e-13)
+    Q = g.standard_normal((M, d))
+    Keq = np.tile(g.standard_normal((1, d)), (N, 1))
+    np.testing.assert_allclose(oracle.cap_scores(Q, Keq), M / N, rtol=1e-13)
+
+
+def test_single_key_takes_everything():
+    g = rnd(3)
+    Q = g.standard_normal((9, 32))
+    np.testing.assert_allclose(oracle.cap_scores(Q, g.standard_normal((1, 32))), [9.0], rtol=1e-14)
+
+
+def test_dominant_key_limit():
+    g = rnd(4)
+    d, N = 16, 50
+    q = g.standard_normal((1, d))
+    K = g.standard_normal((N, d))
+    K[17] = 200.0 * q[0]
+    u = oracle.cap_scores(q, K)
+    assert u[17] > 1 - 1e-12 and abs(u.sum() - 1) < 1e-12
+
+
+def test_key_shift_invariance():
+    # adding one vector c to every key adds q.c/sqrt(d) to a whole row: softmax unchanged
+    g = rnd(5)
+    Q, K = g.standard_normal((8, 24)), g.standard_normal((70, 24))
+    c = g.standard_normal((1, 24)) * 5
+    np.testing.assert_allclose(oracle.cap_scores(Q, K + c), oracle.cap_scores(Q, K), rtol=1e-9)
+
+
+def test_slot_permutation_equivariance():
+    g = rnd(6)
+    Q, K = g.standard_normal((8, 24)), g.standard_normal((70, 24))
+    perm = g.permutation(70)
+    np.testing.assert_allclose(oracle.cap_scores(Q, K[perm]), oracle.cap_scores(Q, K)[perm], rtol=1e-12)
+
+
+def test_row_order_does_not_matter_but_rows_add():
+    g = rnd(7)
+    Q, K = g.standard_normal((6, 8)), g.standard_normal((20, 8))
+    whole = oracle.cap_scores(Q, K)
+    parts = sum(oracle.cap_scores(Q[i:i + 1], K) for i in range(6))
+    np.testing.assert_allclose(whole, parts, rtol=1e-13)
+
+
+def test_single_row_is_a_library_softmax():
+    torch = pytest.importorskip("torch")
+    from scipy.special import softmax
+    g = rnd(8)
+    d = 64
+    q, K = g.standard_normal((1, d)), g.standard_normal((300, d))
+    u = oracle.cap_scores(q, K)
+    logits = (K @ q[0]) / np.sqrt(d)
+    np.testing.assert_allclose(u, softmax(logits), rtol=1e-12)
+    t = torch.softmax(torch.from_numpy(logits), dim=0).numpy()
+    np.testing.assert_allclose(u, t, rtol=1e-12)
+
+
+def test_many_rows_against_library_softmax():
+    from scipy.special import softmax
+    g = rnd(9)
+    d = 32
+    Q, K = g.standard_normal((12, d)) * 2, g.standard_normal((90, d)) * 2
+    ref = softmax(Q @ K.T / np.sqrt(d), axis=1).sum(axis=0)
+    np.testing.assert_allclose(oracle.cap_scores(Q, K), ref, rtol=1e-12)
+
+
+def test_scale_is_one_over_sqrt_d():
+    # d = 16: logits are q.k/4.  One row, two keys, q.k = (0, 4 ln 3) -> p = (1/4, 3/4)
+    d = 16
+    q = np.zeros((1, d)); q[0, 0] = 1.0
+    K = np.zeros((2, d)); K[1, 0] = 4 * np.log(3.0)
+    np.testing.assert_allclose(oracle.cap_scores(q, K), [0.25, 0.75], rtol=1e-14)
+
+
+# ---------------------------------------------------------------- selection
+def brute_best_subset(vals, cand, r):
+    best, arg = None, None
+    for sub in itertools.combinations(cand, r):
+        s = sum(vals[j] for j in sub)
+        if best is None or s > best:
+            best, arg = s, sub
+    return set(arg) if arg is not None else set()
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_selection_is_the_brute_force_maximiser(seed):
+    g = rnd(100 + seed)
+    N = int(g.integers(4, 13))
+    keep = int(g.integers(1, N))
+    T = int(g.integers(0, keep + 1))
+    aux, u = g.random(N), g.random(N)
+    nuc = oracle.nuc_top(aux, T)
+    assert set(nuc.tolist()) == brute_best_subset(aux, range(N), T)
+    assert list(nuc) == sorted(nuc)
+    idx = oracle.select(u, nuc, keep)
+    rest = [j for j in range(N) if j not in set(nuc.tolist())]
+    want = set(nuc.tolist()) | brute_best_subset(u, rest, keep - T)
+    assert set(idx.tolist()) == want
+    assert len(idx) == keep and list(idx) == sorted(set(idx.tolist()))
+
+
+def test_selection_invariants_large():
+    g = rnd(20)
+    N, keep, T = 1000, 400, 150
+    aux, u = g.random(N), g.random(N)
+    nuc = oracle.nuc_top(aux, T)
+    idx = oracle.select(u, nuc, keep)
+    assert len(idx) == keep and (np.diff(idx) > 0).all()
+    assert set(nuc.tolist()) <= set(idx.tolist())
+    assert aux[nuc].min() >= np.delete(aux, nuc).max()
+    kept_cap = np.setdiff1d(idx, nuc)
+    dropped = np.setdiff1d(np.arange(N), idx)
+    assert len(kept_cap) == keep - T
+    assert u[kept_cap].min() >= u[dropped].max()
+
+
+def test_nuc_only_and_cap_only_special_cases():
+    g = rnd(21)
+    N, keep = 200, 60
+    aux = g.random(N)
+    # T = keep: every head keeps the same slots whatever its CaP scores (NuC is per token)
+    nuc = oracle.nuc_top(aux, keep)
+    a = oracle.select(g.random(N), nuc, keep)
+    b = oracle.select(g.random(N), nuc, keep)
+    assert (a == b).all() and (a == nuc).all()
+    # T = 0: plain top-k of the CaP score (library sort as the reference)
+    u = g.random(N)
+    idx = oracle.select(u, np.empty(0, dtype=np.int32), keep)
+    assert set(idx.tolist()) == set(np.argsort(-u, kind="stable")[:keep].tolist())
+
+
+def test_fill_with_max_then_one_topk_gives_the_same_set():
+    # Appendix B combines the two scores by raising the NuC slots to the tensor's
+    # maximum and taking a single top-|C|; Sec. 3.3.3 describes two separate
+    # rankings.  With at least one CaP slot and distinct scores they agree.
+    g = rnd(22)
+    N, keep, T = 300, 120, 50
+    aux, u = g.random(N), g.random(N)
+    nuc = oracle.nuc_top(aux, T)
+    filled = u.copy()
+    filled[nuc] = np.inf  # strictly above every CaP score: the NuC slots can never lose
+    one_topk = set(np.argsort(-filled, kind="stable")[:keep].tolist())
+    assert set(oracle.select(u, nuc, keep).tolist()) == one_topk
+
+
+def test_ties_prefer_lower_slots():
+    N = 50
+    nuc = oracle.nuc_top(np.ones(N), 7)
+    assert nuc.tolist() == list(range(7))
+    idx = oracle.select(np.full(N, 0.5), nuc, 20)
+    assert idx.tolist() == list(range(20))
+    u = np.zeros(N); u[40:] = 1.0
+    idx = oracle.select(u, np.array([3], dtype=np.int32), 13)
+    assert idx.tolist() == [0, 1, 3] + list(range(40, 50))
+
+
+# ---------------------------------------------------------------- gather
+def test_gather_is_bytewise_row_copy():
+    g = rnd(30)
+    rows = g.integers(0, 65536, size=(64, 24), dtype=np.uint16)
+    idx = np.sort(g.choice(64, 20, replace=False)).astype(np.int32)
+    out = oracle.gather(rows, idx)
+    assert out.dtype == rows.dtype and (out == rows[idx]).all()
+    ident = oracle.gather(rows, np.arange(64, dtype=np.int32))
+    assert (ident == rows).all()
+
+
+# ---------------------------------------------------------------- whole cycle wiring
+def test_cycle_wiring_gqa_streams_layers():
+    g = rnd(40)
+    L, B, Hq, Hkv, P, d, N, keep, T = 2, 3, 6, 2, 4, 8, 30, 12, 5
+    G = Hq // Hkv
+    Q = g.standard_normal((L, B, Hq, P, d)).astype(np.float32)
+    K = g.standard_normal((L, B, Hkv, N, d)).astype(np.float32)
+    V = g.standard_normal((L, B, Hkv, N, d)).astype(np.float32)
+    aux = g.random((B, N)).astype(np.float32)
+    out = oracle.cycle(Q, K, V, aux, keep, T)
+    assert out["u"].shape == (L * B * Hkv, N)
+    for l in range(L):
+        for b in range(B):
+            nuc = oracle.nuc_top(aux[b], T)
+            for kv in range(Hkv):
+                unit = (l * B + b) * Hkv + kv
+                # query head h serves kv head h // G; its P rows add to the same score
+                u = sum(oracle.cap_scores(Q[l, b, h].astype(np.float64), K[l, b, kv].astype(np.float64))
+                        for h in range(Hq) if h // G == kv)
+                np.testing.assert_allclose(out["u"][unit], u, rtol=1e-12)
+                assert abs(out["u"][unit].sum() - G * P) < 1e-9
+                idx = oracle.select(out["u"][unit], nuc, keep)
+                assert (out["idx"][unit] == idx).all()
+                assert (out["K"][unit] == K[l, b, kv][idx]).all()
+                assert (out["V"][unit] == V[l, b, kv][idx]).all()
+    # a subset of units gives the same rows
+    sub = oracle.cycle(Q, K, V, aux, keep, T, units=[7, 2])
+    assert (sub["idx"][0] == out["idx"][7]).all() and (sub["idx"][1] == out["idx"][2]).all()
+    np.testing.assert_array_equal(sub["u"][1], out["u"][2])
+
+
+def test_cycle_accepts_bf16_bit_patterns():
+    torch = pytest.importorskip("torch")
+    g = rnd(41)
+    x = g.standard_normal((1, 1, 2, 3, 8)).astype(np.float32)
+    bits = torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    wide = oracle.widen_storage(bits)
+    assert (wide == torch.from_numpy(x).to(torch.bfloat16).to(torch.float64).numpy()).all()
