@@ -1,0 +1,181 @@
+/*
+ * ipot.h - C ABI of the memory-pot library: the Continual Context Distillation
+ * (CCD) compression cycle of InfiniPot (arxiv 2410.01518) on one CUDA device.
+ *
+ * The pot is the paper's fixed-size KV cache (Sec. 3.1: at most |M| entries;
+ * Sec. 3.2: filled sequentially, then distilled to |C| entries, then filled
+ * again).  One pot object holds, for every (layer, stream, kv-head) "unit", a
+ * K and a V array of pot_size rows of d elements.
+ *
+ * Memory layouts (all dense, row-major, innermost index last):
+ *   pot K, V     [layers][batch][Hkv][pot_size][d]   element = bf16 or f32
+ *   chunk K, V   [layers][batch][Hkv][n_tokens][d]   same element type
+ *   Q_cap        [layers][batch][Hq][cap_rows][d]    same element type
+ *   aux_scores   [batch][len]                        f32, higher = more novel
+ *   scores       [layers][batch][Hkv][len]           f32
+ *   indices      [layers][batch][Hkv][keep]          int32, strictly ascending
+ * Query head h attends to KV head h / (Hq / Hkv).
+ *
+ * Conventions
+ *   - Every function returns IPOT_OK (0) or a negative IPOT_E_* code; nothing
+ *     is thrown across the boundary.  ipot_strerror() names a code.
+ *   - Argument and state errors are found on the host before anything is
+ *     launched and leave the pot unchanged.
+ *   - Unless a function's name ends in _host, its data pointers are DEVICE
+ *     pointers on the pot's device, 16-byte aligned, owned by the caller and
+ *     only read.  Work is queued on the pot's stream and the call returns
+ *     without waiting; the caller must keep the buffers alive and unchanged
+ *     until that work has run (synchronise the stream or call
+ *     ipot_sync_status()).
+ *   - The library owns the pot, the score/index arrays and its scratch; they
+ *     are allocated in ipot_create*() and freed in ipot_destroy().
+ *   - A pot object is not thread-safe; use one host thread per pot at a time.
+ *   - There is no CPU fallback: without a usable CUDA device every call that
+ *     touches data fails with IPOT_E_CUDA.
+ */
+#ifndef IPOT_H
+#define IPOT_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ipot ipot_t; /* opaque, library-owned */
+
+enum {
+    IPOT_OK = 0,
+    IPOT_E_INVALID = -1, /* bad argument (NULL, misaligned, out of range, unsupported shape) */
+    IPOT_E_STATE = -2,   /* call not allowed in the pot's current state (overflow, nothing to distil) */
+    IPOT_E_NOMEM = -3,   /* device or host allocation failed */
+    IPOT_E_CUDA = -4,    /* a CUDA runtime/driver call failed, or no device */
+    IPOT_E_TIMEOUT = -5, /* a bounded device-side wait gave up (sticky, reported by ipot_sync_status) */
+    IPOT_E_BOUNDS = -6   /* a device-side self-check found an index out of range (sticky) */
+};
+
+enum { IPOT_BF16 = 0, IPOT_F32 = 1 };
+
+/* Which scoring kernel ipot_score_and_compress() uses. */
+enum {
+    IPOT_SCORER_AUTO = 0,   /* tensor-core kernel when the shape allows it, else the SIMT kernel */
+    IPOT_SCORER_SIMT = 1,   /* fp32 FMA kernel: any supported shape, f32 or bf16 */
+    IPOT_SCORER_TENSOR = 2  /* tcgen05 kernel: IPOT_E_INVALID if the shape does not allow it */
+};
+
+typedef struct {
+    int pot_size;     /* context slots per unit (the paper's |M| minus the CaP rows) */
+    int keep;         /* |C|: entries that survive a cycle, 0 < keep < pot_size */
+    int layers, Hq, Hkv, d;
+    int batch;        /* independent streams, >= 1 */
+    int dtype;        /* IPOT_BF16 or IPOT_F32 */
+    int nuc_slots;    /* T of Sec. 3.3.3, 0 <= T <= keep; -1 = keep / 2 (the 50 % ratio of Sec. 4.4.2) */
+    int max_cap_rows; /* largest cap_rows that will be passed (scratch is sized for it) */
+    void *stream;     /* cudaStream_t, NULL = the default stream */
+} ipot_config_t;
+
+/*
+ * Sec. 3.1-3.2: create an empty pot (len = 0) on the current CUDA device with
+ * batch = 1, bf16 elements, T = keep / 2, up to 64 CaP rows, default stream.
+ * Limits: Hq % Hkv == 0; d a multiple of 8 with 32 <= d <= 256; 0 < keep <
+ * pot_size <= 32768.  *out is set only on success.  Errors: INVALID, NOMEM, CUDA.
+ */
+int ipot_create(int pot_size, int keep, int layers, int Hq, int Hkv, int d, ipot_t **out);
+
+/* Same, with every parameter explicit. */
+int ipot_create_ex(const ipot_config_t *cfg, ipot_t **out);
+
+/* Waits for the pot's queued work, frees everything.  NULL is accepted. */
+int ipot_destroy(ipot_t *pot);
+
+/* Use another cudaStream_t for all later calls (the caller orders the hand-over). */
+int ipot_set_stream(ipot_t *pot, void *cuda_stream);
+
+/* Sec. 3.3.3 / Sec. 4.4.2: number of slots T given to the novelty ranking, 0 <= T <= keep. */
+int ipot_set_nuc_slots(ipot_t *pot, int T);
+
+/* IPOT_SCORER_*; TENSOR is refused at the next cycle if the shape does not allow it. */
+int ipot_set_scorer(ipot_t *pot, int scorer);
+
+/* Forget the contents: len = 0.  Nothing is launched. */
+int ipot_reset(ipot_t *pot);
+
+/*
+ * Sec. 3.2 ("filling the remaining cache space sequentially"): copy n_tokens
+ * new rows of every unit behind the rows already in the pot; len += n_tokens.
+ * K, V: device, [layers][batch][Hkv][n_tokens][d].
+ * Errors: INVALID (NULL, misaligned, n_tokens <= 0), STATE (len + n_tokens >
+ * pot_size; the pot is unchanged), CUDA.
+ */
+int ipot_append_chunk(ipot_t *pot, const void *K, const void *V, int n_tokens);
+
+/* Same with HOST buffers (pinned memory makes the copy asynchronous): the
+ * rows go straight from host memory into the pot with strided copies. */
+int ipot_append_chunk_host(ipot_t *pot, const void *K_host, const void *V_host, int n_tokens);
+
+/*
+ * One CCD cycle (Sec. 3.2) over all units, N = len rows in the pot:
+ *   1. Sec. 3.3.3: per stream, the T slots with the largest aux_scores are
+ *      reserved in every head (ties: lower slot first);
+ *   2. Sec. 3.3.1, Eq. 2: per unit, u_j = sum over the G*cap_rows query rows of
+ *      the unit's KV head of softmax_j(q . k_j / sqrt(d)), the softmax taken
+ *      over the N pot keys; fp32 arithmetic, probabilities never stored;
+ *   3. Sec. 3.3.3 / Appendix B: per unit, the keep - T non-reserved slots with
+ *      the largest u_j join the reserved ones (ties: lower slot first);
+ *   4. Appendix B: K and V rows of the survivors are moved, in place and in
+ *      their original order, to rows 0 .. keep-1; len = keep.
+ * Q_cap: device [layers][batch][Hq][cap_rows][d]; aux_scores: device
+ * [batch][len] f32, may be NULL iff T == 0.  All inputs must be finite.
+ * Errors: INVALID (NULL, misaligned, cap_rows < 1 or > max_cap_rows, scorer
+ * not applicable), STATE (len <= keep: nothing to distil; pot unchanged), CUDA.
+ */
+int ipot_score_and_compress(ipot_t *pot, const void *Q_cap, int cap_rows, const float *aux_scores);
+
+/*
+ * Same with HOST buffers: Q_cap_host and aux_host are copied to library-owned
+ * device staging first; if idx_host is not NULL the index lists
+ * ([layers][batch][Hkv][keep] int32) are copied back into it.  All copies are
+ * queued on the pot's stream; with pageable memory they block the caller.
+ */
+int ipot_score_and_compress_host(ipot_t *pot, const void *Q_cap_host, int cap_rows,
+                                 const float *aux_host, int32_t *idx_host);
+
+/* Steps 1-2 of the cycle only: fills the score array, leaves the pot and len
+ * untouched (aux_scores may be NULL: step 1 is then skipped). */
+int ipot_score_only(ipot_t *pot, const void *Q_cap, int cap_rows, const float *aux_scores);
+
+/*
+ * Borrowed device pointers to the pot ([layers][batch][Hkv][pot_size][d]) and
+ * the current fill.  Rows >= len are undefined.  The pointers stay valid until
+ * ipot_destroy(); their contents are final once the stream's queued work ran.
+ * Any of K, V, len may be NULL.
+ */
+int ipot_view(ipot_t *pot, void **K, void **V, int *len);
+
+/* Results of the last cycle (device, library-owned, overwritten by the next cycle). */
+int ipot_last_indices(ipot_t *pot, const int32_t **idx);            /* [layers][batch][Hkv][keep] */
+int ipot_last_scores(ipot_t *pot, const float **u, int *len_before); /* [layers][batch][Hkv][len_before] */
+
+/* Waits for the pot's stream and returns the sticky device status
+ * (IPOT_OK, IPOT_E_TIMEOUT, IPOT_E_BOUNDS) or IPOT_E_CUDA. */
+int ipot_sync_status(ipot_t *pot);
+
+/*
+ * Per-kernel device timing.  When enabled, every cycle records CUDA events on
+ * the pot's stream around its kernels; ipot_last_kernel_ms() waits for the last
+ * cycle and returns, in milliseconds: ms[0] NuC ranking, ms[1] CaP scoring,
+ * ms[2] per-head selection, ms[3] K/V compaction.  *scorer_used (may be NULL)
+ * receives IPOT_SCORER_SIMT or IPOT_SCORER_TENSOR.
+ */
+int ipot_set_profiling(ipot_t *pot, int on);
+int ipot_last_kernel_ms(ipot_t *pot, float ms[4], int *scorer_used);
+
+/* Number of kernels this pot has launched since it was created. */
+int ipot_launch_count(ipot_t *pot, long long *launches);
+
+const char *ipot_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* IPOT_H */

@@ -1,0 +1,435 @@
+// Host side of the memory-pot library: pot state, argument checks, launches.
+// The C ABI is declared and documented in include/ipot.h.
+#include "../../include/ipot.h"
+
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "common.cuh"
+#include "k_move.cuh"
+#include "k_score_simt.cuh"
+#include "k_score_tc.cuh"
+#include "k_select.cuh"
+
+using namespace ipotk;
+
+struct ipot {
+    ipot_config_t cfg;
+    int len;
+    int device;
+    int sm_count;
+    int scorer;
+    int G, units, elem_bytes, row_bytes;
+    cudaStream_t stream;
+    // device memory (library-owned)
+    void *K, *V;
+    float *scores;       // [max_parts][units * pot_size]; array q holds [units][N] partial scores of the
+                         // q-th block of 128 query rows (the SIMT scorer writes array 0 only)
+    float *summed;       // [units][N]: sum of the partial arrays when there are several
+    int max_parts;
+    float2 *row_stats;   // [units][max M]
+    uint8_t *nuc_mask;   // [batch][pot_size]
+    int32_t *idx;        // [units][keep]
+    int *status;         // sticky device status word
+    void *stage_q;       // device staging for the *_host calls
+    float *stage_aux;
+    // results of the last cycle
+    int last_len_before;
+    const float *last_scores;
+    int last_scorer;
+    // timing
+    int profiling;
+    cudaEvent_t ev[5];
+    bool ev_valid;
+    long long launches;
+    TcPlan tc;           // tensor-core scorer state
+};
+
+namespace {
+
+#define IPOT_CUDA(call)                                                             \
+    do {                                                                            \
+        cudaError_t e_ = (call);                                                    \
+        if (e_ != cudaSuccess) {                                                    \
+            if (getenv("IPOT_DEBUG"))                                               \
+                fprintf(stderr, "ipot: %s -> %s\n", #call, cudaGetErrorString(e_)); \
+            return IPOT_E_CUDA;                                                     \
+        }                                                                           \
+    } while (0)
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_config(const ipot_config_t &c)
+{
+    if (c.pot_size <= 0 || c.pot_size > 32768) return IPOT_E_INVALID;
+    if (c.keep <= 0 || c.keep >= c.pot_size) return IPOT_E_INVALID;
+    if (c.layers <= 0 || c.batch <= 0 || c.Hq <= 0 || c.Hkv <= 0 || c.Hq % c.Hkv) return IPOT_E_INVALID;
+    if (c.d < 32 || c.d > 256 || c.d % 8) return IPOT_E_INVALID;
+    if (c.dtype != IPOT_BF16 && c.dtype != IPOT_F32) return IPOT_E_INVALID;
+    if (c.nuc_slots < -1 || c.nuc_slots > c.keep) return IPOT_E_INVALID;
+    if (c.max_cap_rows <= 0 || c.max_cap_rows > 4096) return IPOT_E_INVALID;
+    return IPOT_OK;
+}
+
+void free_all(ipot *p)
+{
+    tc_plan_destroy(p->tc);
+    cudaFree(p->K); cudaFree(p->V); cudaFree(p->scores); cudaFree(p->summed);
+    cudaFree(p->row_stats); cudaFree(p->nuc_mask); cudaFree(p->idx); cudaFree(p->status);
+    cudaFree(p->stage_q); cudaFree(p->stage_aux);
+    for (auto &e : p->ev) if (e) cudaEventDestroy(e);
+}
+
+template <typename T>
+int launch_simt(ipot *p, const void *Q, int M, int N)
+{
+    const int d = p->cfg.d;
+    const size_t smem = simt_smem_bytes(d);
+    IPOT_CUDA(cudaFuncSetAttribute(cap_row_stats<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)simt_smem_bytes(256)));
+    IPOT_CUDA(cudaFuncSetAttribute(cap_column_sums<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)simt_smem_bytes(256)));
+    const float scale_log2e = (float)(1.4426950408889634 / std::sqrt((double)d));
+    const size_t kstride = (size_t)p->cfg.pot_size * d;
+    dim3 g1((M + kSimtRows - 1) / kSimtRows, p->units), g2((N + kSimtKeys - 1) / kSimtKeys, p->units);
+    cap_row_stats<T><<<g1, kSimtThreads, smem, p->stream>>>((const T *)Q, (const T *)p->K, p->row_stats, M, N, d, kstride, scale_log2e);
+    cap_column_sums<T><<<g2, kSimtThreads, smem, p->stream>>>((const T *)Q, (const T *)p->K, p->row_stats, p->scores, M, N, d, kstride, scale_log2e);
+    p->launches += 2;
+    IPOT_CUDA(cudaGetLastError());
+    return IPOT_OK;
+}
+
+// Steps 1-2 (and the timing events around them).  On success *parts tells how many
+// partial score arrays the scorer wrote.
+int run_scoring(ipot *p, const void *Q, int cap_rows, const float *aux, int *parts)
+{
+    const int N = p->len, T = p->cfg.nuc_slots, M = p->G * cap_rows;
+    int scorer = p->scorer;
+    const bool tc_ok = tc_applicable(p->tc, p->cfg, N, M);
+    if (scorer == IPOT_SCORER_TENSOR && !tc_ok) return IPOT_E_INVALID;
+    if (scorer == IPOT_SCORER_AUTO) scorer = tc_ok ? IPOT_SCORER_TENSOR : IPOT_SCORER_SIMT;
+
+    if (p->profiling) IPOT_CUDA(cudaEventRecord(p->ev[0], p->stream));
+    if (T > 0 && aux) {
+        IPOT_CUDA(cudaFuncSetAttribute(nuc_mask_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 32768 * 4));
+        nuc_mask_kernel<<<p->cfg.batch, kSelThreads, (size_t)N * 4, p->stream>>>(aux, p->nuc_mask, N, T);
+        p->launches += 1;
+        IPOT_CUDA(cudaGetLastError());
+    }
+    if (p->profiling) IPOT_CUDA(cudaEventRecord(p->ev[1], p->stream));
+    *parts = 1;
+    int rc;
+    if (scorer == IPOT_SCORER_TENSOR) {
+        int n_launch = 0;
+        rc = tc_launch(p->tc, p->cfg, Q, p->K, p->scores, (size_t)p->units * p->cfg.pot_size, N, M, p->units, p->status,
+                       p->stream, parts, &n_launch);
+        p->launches += n_launch;
+    } else {
+        rc = p->cfg.dtype == IPOT_F32 ? launch_simt<float>(p, Q, M, N) : launch_simt<__nv_bfloat16>(p, Q, M, N);
+    }
+    if (rc != IPOT_OK) return rc;
+    if (p->profiling) IPOT_CUDA(cudaEventRecord(p->ev[2], p->stream));
+    p->last_scorer = scorer;
+    p->last_len_before = N;
+    p->last_scores = (*parts > 1) ? p->summed : p->scores;
+    return IPOT_OK;
+}
+
+int check_cycle_args(ipot *p, const void *Q, int cap_rows, const float *aux, bool compress)
+{
+    if (!p || !Q) return IPOT_E_INVALID;
+    if (cap_rows < 1 || cap_rows > p->cfg.max_cap_rows) return IPOT_E_INVALID;
+    if (compress && p->cfg.nuc_slots > 0 && !aux) return IPOT_E_INVALID;
+    if (compress ? (p->len <= p->cfg.keep) : (p->len < 1)) return IPOT_E_STATE;
+    return IPOT_OK;
+}
+
+int compact_slices(const ipot *p)
+{
+    const int row_vecs = p->row_bytes / 16;
+    const char *env = getenv("IPOT_COMPACT_SLICES");
+    const int want = env ? atoi(env) : 0;
+    if (want > 0 && row_vecs % want == 0) return want;
+    int slices = 1;
+    while (row_vecs % (slices * 2) == 0 && row_vecs / (slices * 2) >= 4 &&
+           (long long)p->units * 2 * slices < 8LL * p->sm_count)
+        slices *= 2;
+    return slices;
+}
+
+int run_cycle(ipot *p, const void *Q, int cap_rows, const float *aux)
+{
+    const int N = p->len, keep = p->cfg.keep, T = p->cfg.nuc_slots;
+    int parts = 1;
+    int rc = run_scoring(p, Q, cap_rows, aux, &parts);
+    if (rc != IPOT_OK) return rc;
+    const size_t part_stride = (size_t)p->units * p->cfg.pot_size;
+    IPOT_CUDA(cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 32768 * 4));
+    select_kernel<<<p->units, kSelThreads, (size_t)N * 4, p->stream>>>(
+        p->scores, parts, part_stride, T > 0 ? p->nuc_mask : nullptr, p->idx,
+        parts > 1 ? p->summed : nullptr, N, keep, p->cfg.Hkv, p->cfg.batch, p->status);
+    p->launches += 1;
+    IPOT_CUDA(cudaGetLastError());
+    if (p->profiling) IPOT_CUDA(cudaEventRecord(p->ev[3], p->stream));
+
+    const int row_vecs = p->row_bytes / 16;
+    const int slices = compact_slices(p);
+    dim3 grid(slices, p->units, 2);
+    compact_kernel<<<grid, kMoveThreads, 0, p->stream>>>((uint4 *)p->K, (uint4 *)p->V, p->idx, keep, N, row_vecs,
+                                                        row_vecs / slices, (size_t)p->cfg.pot_size * row_vecs, p->status);
+    p->launches += 1;
+    IPOT_CUDA(cudaGetLastError());
+    if (p->profiling) {
+        IPOT_CUDA(cudaEventRecord(p->ev[4], p->stream));
+        p->ev_valid = true;
+    }
+    p->len = keep;
+    return IPOT_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int ipot_create(int pot_size, int keep, int layers, int Hq, int Hkv, int d, ipot_t **out)
+{
+    ipot_config_t c;
+    memset(&c, 0, sizeof(c));
+    c.pot_size = pot_size; c.keep = keep; c.layers = layers; c.Hq = Hq; c.Hkv = Hkv; c.d = d;
+    c.batch = 1; c.dtype = IPOT_BF16; c.nuc_slots = -1; c.max_cap_rows = 64; c.stream = nullptr;
+    return ipot_create_ex(&c, out);
+}
+
+int ipot_create_ex(const ipot_config_t *cfg, ipot_t **out)
+{
+    if (!cfg || !out) return IPOT_E_INVALID;
+    int rc = check_config(*cfg);
+    if (rc != IPOT_OK) return rc;
+    ipot *p = new (std::nothrow) ipot();
+    if (!p) return IPOT_E_NOMEM;
+    p->cfg = *cfg;
+    if (p->cfg.nuc_slots < 0) p->cfg.nuc_slots = p->cfg.keep / 2;
+    p->G = cfg->Hq / cfg->Hkv;
+    p->units = cfg->layers * cfg->batch * cfg->Hkv;
+    p->elem_bytes = cfg->dtype == IPOT_F32 ? 4 : 2;
+    p->row_bytes = cfg->d * p->elem_bytes;
+    p->stream = (cudaStream_t)cfg->stream;
+    p->scorer = IPOT_SCORER_AUTO;
+    if (cudaGetDevice(&p->device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, p->device) != cudaSuccess) {
+        cudaGetLastError();
+        delete p;
+        return IPOT_E_CUDA;
+    }
+    const size_t pot_bytes = (size_t)p->units * cfg->pot_size * p->row_bytes;
+    const int maxM = p->G * cfg->max_cap_rows;
+    p->max_parts = (maxM + 127) / 128;
+    const size_t score_elems = (size_t)p->units * cfg->pot_size;
+    bool ok = true;
+    auto alloc = [&](void **ptr, size_t bytes) {
+        if (ok && cudaMalloc(ptr, bytes ? bytes : 16) != cudaSuccess) ok = false;
+    };
+    alloc(&p->K, pot_bytes);
+    alloc(&p->V, pot_bytes);
+    alloc((void **)&p->scores, score_elems * 4 * p->max_parts);
+    alloc((void **)&p->summed, score_elems * 4);
+    alloc((void **)&p->row_stats, (size_t)p->units * maxM * sizeof(float2));
+    alloc((void **)&p->nuc_mask, (size_t)cfg->batch * cfg->pot_size);
+    alloc((void **)&p->idx, (size_t)p->units * cfg->keep * 4);
+    alloc((void **)&p->status, 16);
+    alloc(&p->stage_q, (size_t)p->units * maxM * p->row_bytes);
+    alloc((void **)&p->stage_aux, (size_t)cfg->batch * cfg->pot_size * 4);
+    if (ok) ok = cudaMemset(p->status, 0, 16) == cudaSuccess;
+    for (auto &e : p->ev)
+        if (ok && cudaEventCreate(&e) != cudaSuccess) ok = false;
+    if (!ok) {
+        cudaGetLastError();
+        free_all(p);
+        delete p;
+        return IPOT_E_NOMEM;
+    }
+    tc_plan_init(p->tc, p->cfg, p->K, p->sm_count);
+    *out = p;
+    return IPOT_OK;
+}
+
+int ipot_destroy(ipot_t *p)
+{
+    if (!p) return IPOT_OK;
+    cudaStreamSynchronize(p->stream);
+    free_all(p);
+    delete p;
+    return IPOT_OK;
+}
+
+int ipot_set_stream(ipot_t *p, void *s)
+{
+    if (!p) return IPOT_E_INVALID;
+    p->stream = (cudaStream_t)s;
+    return IPOT_OK;
+}
+
+int ipot_set_nuc_slots(ipot_t *p, int T)
+{
+    if (!p || T < 0 || T > p->cfg.keep) return IPOT_E_INVALID;
+    p->cfg.nuc_slots = T;
+    return IPOT_OK;
+}
+
+int ipot_set_scorer(ipot_t *p, int scorer)
+{
+    if (!p || scorer < IPOT_SCORER_AUTO || scorer > IPOT_SCORER_TENSOR) return IPOT_E_INVALID;
+    p->scorer = scorer;
+    return IPOT_OK;
+}
+
+int ipot_reset(ipot_t *p)
+{
+    if (!p) return IPOT_E_INVALID;
+    p->len = 0;
+    return IPOT_OK;
+}
+
+int ipot_append_chunk(ipot_t *p, const void *K, const void *V, int n)
+{
+    if (!p || !K || !V || n <= 0 || !aligned16(K) || !aligned16(V)) return IPOT_E_INVALID;
+    if (p->len + n > p->cfg.pot_size) return IPOT_E_STATE;
+    const size_t row_vecs = p->row_bytes / 16;
+    const size_t n_vecs = (size_t)n * row_vecs;
+    int pieces = (int)((n_vecs + (size_t)kMoveThreads * kMoveVecs - 1) / ((size_t)kMoveThreads * kMoveVecs));
+    if (pieces < 1) pieces = 1;
+    dim3 grid(pieces, p->units, 2);
+    append_kernel<<<grid, kMoveThreads, 0, p->stream>>>((const uint4 *)K, (const uint4 *)V, (uint4 *)p->K, (uint4 *)p->V,
+                                                       n_vecs, (size_t)p->cfg.pot_size * row_vecs, (size_t)p->len * row_vecs);
+    p->launches += 1;
+    IPOT_CUDA(cudaGetLastError());
+    p->len += n;
+    return IPOT_OK;
+}
+
+int ipot_append_chunk_host(ipot_t *p, const void *K, const void *V, int n)
+{
+    if (!p || !K || !V || n <= 0) return IPOT_E_INVALID;
+    if (p->len + n > p->cfg.pot_size) return IPOT_E_STATE;
+    const size_t width = (size_t)n * p->row_bytes, dpitch = (size_t)p->cfg.pot_size * p->row_bytes;
+    char *dK = (char *)p->K + (size_t)p->len * p->row_bytes, *dV = (char *)p->V + (size_t)p->len * p->row_bytes;
+    IPOT_CUDA(cudaMemcpy2DAsync(dK, dpitch, K, width, width, p->units, cudaMemcpyHostToDevice, p->stream));
+    IPOT_CUDA(cudaMemcpy2DAsync(dV, dpitch, V, width, width, p->units, cudaMemcpyHostToDevice, p->stream));
+    p->len += n;
+    return IPOT_OK;
+}
+
+int ipot_score_and_compress(ipot_t *p, const void *Q, int cap_rows, const float *aux)
+{
+    int rc = check_cycle_args(p, Q, cap_rows, aux, true);
+    if (rc != IPOT_OK) return rc;
+    if (!aligned16(Q) || (aux && (reinterpret_cast<uintptr_t>(aux) & 3u))) return IPOT_E_INVALID;
+    return run_cycle(p, Q, cap_rows, aux);
+}
+
+int ipot_score_and_compress_host(ipot_t *p, const void *Q, int cap_rows, const float *aux, int32_t *idx_host)
+{
+    int rc = check_cycle_args(p, Q, cap_rows, aux, true);
+    if (rc != IPOT_OK) return rc;
+    const size_t qbytes = (size_t)p->units * p->G * cap_rows * p->row_bytes;
+    IPOT_CUDA(cudaMemcpyAsync(p->stage_q, Q, qbytes, cudaMemcpyHostToDevice, p->stream));
+    if (aux) IPOT_CUDA(cudaMemcpyAsync(p->stage_aux, aux, (size_t)p->cfg.batch * p->len * 4, cudaMemcpyHostToDevice, p->stream));
+    rc = run_cycle(p, p->stage_q, cap_rows, aux ? p->stage_aux : nullptr);
+    if (rc != IPOT_OK) return rc;
+    if (idx_host)
+        IPOT_CUDA(cudaMemcpyAsync(idx_host, p->idx, (size_t)p->units * p->cfg.keep * 4, cudaMemcpyDeviceToHost, p->stream));
+    return IPOT_OK;
+}
+
+int ipot_score_only(ipot_t *p, const void *Q, int cap_rows, const float *aux)
+{
+    int rc = check_cycle_args(p, Q, cap_rows, aux, false);
+    if (rc != IPOT_OK) return rc;
+    if (!aligned16(Q)) return IPOT_E_INVALID;
+    int parts = 1;
+    rc = run_scoring(p, Q, cap_rows, aux, &parts);
+    if (rc != IPOT_OK) return rc;
+    if (parts > 1) {
+        const size_t n = (size_t)p->units * p->len;
+        sum_parts_kernel<<<(unsigned)((n + 255) / 256), 256, 0, p->stream>>>(
+            p->scores, parts, (size_t)p->units * p->cfg.pot_size, p->summed, n);
+        p->launches += 1;
+        IPOT_CUDA(cudaGetLastError());
+    }
+    return IPOT_OK;
+}
+
+int ipot_view(ipot_t *p, void **K, void **V, int *len)
+{
+    if (!p) return IPOT_E_INVALID;
+    if (K) *K = p->K;
+    if (V) *V = p->V;
+    if (len) *len = p->len;
+    return IPOT_OK;
+}
+
+int ipot_last_indices(ipot_t *p, const int32_t **idx)
+{
+    if (!p || !idx) return IPOT_E_INVALID;
+    *idx = p->idx;
+    return IPOT_OK;
+}
+
+int ipot_last_scores(ipot_t *p, const float **u, int *len_before)
+{
+    if (!p || !u) return IPOT_E_INVALID;
+    *u = p->last_scores ? p->last_scores : p->scores;
+    if (len_before) *len_before = p->last_len_before;
+    return IPOT_OK;
+}
+
+int ipot_sync_status(ipot_t *p)
+{
+    if (!p) return IPOT_E_INVALID;
+    IPOT_CUDA(cudaStreamSynchronize(p->stream));
+    int st = 0;
+    IPOT_CUDA(cudaMemcpy(&st, p->status, sizeof(int), cudaMemcpyDeviceToHost));
+    return st;
+}
+
+int ipot_set_profiling(ipot_t *p, int on)
+{
+    if (!p) return IPOT_E_INVALID;
+    p->profiling = on != 0;
+    p->ev_valid = false;
+    return IPOT_OK;
+}
+
+int ipot_last_kernel_ms(ipot_t *p, float ms[4], int *scorer_used)
+{
+    if (!p || !ms) return IPOT_E_INVALID;
+    if (!p->profiling || !p->ev_valid) return IPOT_E_STATE;
+    IPOT_CUDA(cudaEventSynchronize(p->ev[4]));
+    for (int i = 0; i < 4; ++i) IPOT_CUDA(cudaEventElapsedTime(&ms[i], p->ev[i], p->ev[i + 1]));
+    if (scorer_used) *scorer_used = p->last_scorer;
+    return IPOT_OK;
+}
+
+int ipot_launch_count(ipot_t *p, long long *launches)
+{
+    if (!p || !launches) return IPOT_E_INVALID;
+    *launches = p->launches;
+    return IPOT_OK;
+}
+
+const char *ipot_strerror(int code)
+{
+    switch (code) {
+    case IPOT_OK: return "ok";
+    case IPOT_E_INVALID: return "invalid argument";
+    case IPOT_E_STATE: return "call not allowed in the pot's current state";
+    case IPOT_E_NOMEM: return "out of memory";
+    case IPOT_E_CUDA: return "CUDA call failed or no usable device";
+    case IPOT_E_TIMEOUT: return "a bounded device-side wait gave up";
+    case IPOT_E_BOUNDS: return "a device-side self-check found an index out of range";
+    default: return "unknown error code";
+    }
+}
+
+}  // extern "C"

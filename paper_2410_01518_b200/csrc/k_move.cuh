@@ -1,0 +1,75 @@
+// Row movers of the pot:
+//   append_kernel  : Sec. 3.2, "filling the remaining cache space sequentially";
+//   compact_kernel : Appendix B "KV-cache compression" - K'[r] = K[idx[r]],
+//                    V'[r] = V[idx[r]] - done in place.
+// Both move 16-byte vectors.
+#pragma once
+#include "common.cuh"
+
+namespace ipotk {
+
+constexpr int kMoveThreads = 256;
+constexpr int kMoveVecs = 8;  // 16-byte vectors in flight per thread
+
+// grid (pieces, units, 2): tensor z of unit y; src is [units][n_vecs], dst is the pot.
+__global__ void __launch_bounds__(kMoveThreads)
+append_kernel(const uint4 *__restrict__ srcK, const uint4 *__restrict__ srcV, uint4 *__restrict__ potK,
+              uint4 *__restrict__ potV, size_t n_vecs, size_t unit_vecs, size_t first_vec)
+{
+    const uint4 *src = (blockIdx.z ? srcV : srcK) + (size_t)blockIdx.y * n_vecs;
+    uint4 *dst = (blockIdx.z ? potV : potK) + (size_t)blockIdx.y * unit_vecs + first_vec;
+    const size_t stride = (size_t)gridDim.x * kMoveThreads;
+    size_t v = (size_t)blockIdx.x * kMoveThreads + threadIdx.x;
+    for (; v + (kMoveVecs - 1) * stride < n_vecs; v += kMoveVecs * stride) {
+        uint4 t[kMoveVecs];
+#pragma unroll
+        for (int i = 0; i < kMoveVecs; ++i) t[i] = __ldg(src + v + i * stride);
+#pragma unroll
+        for (int i = 0; i < kMoveVecs; ++i) dst[v + i * stride] = t[i];
+    }
+    for (; v < n_vecs; v += stride) dst[v] = __ldg(src + v);
+}
+
+// In-place gather.  grid (slices, units, 2).  A block owns byte columns
+// [slice * slice_vecs, (slice + 1) * slice_vecs) (in 16-byte vectors) of every
+// row of one tensor of one unit, so blocks never touch the same bytes.  idx is
+// ascending, hence idx[r] >= r: the block walks the rows in ascending chunks,
+// reads a whole chunk into registers, synchronises, then writes it.  A chunk's
+// writes land in rows below the next chunk's first row, and every later source
+// row lies at or above it, so nothing that is still needed is overwritten.
+// Rows with idx[r] == r are left alone.
+__global__ void __launch_bounds__(kMoveThreads)
+compact_kernel(uint4 *__restrict__ potK, uint4 *__restrict__ potV, const int32_t *__restrict__ idx,
+               int keep, int N, int row_vecs, int slice_vecs, size_t unit_vecs, int *status)
+{
+    uint4 *base = (blockIdx.z ? potV : potK) + (size_t)blockIdx.y * unit_vecs + (size_t)blockIdx.x * slice_vecs;
+    const int32_t *ix = idx + (size_t)blockIdx.y * keep;
+    const int rows_per_pass = kMoveThreads / slice_vecs;  // rows covered by one vector per thread
+    const int chunk_rows = rows_per_pass * kMoveVecs;
+    const int my_row = threadIdx.x / slice_vecs, my_vec = threadIdx.x - my_row * slice_vecs;
+    for (int r0 = 0; r0 < keep; r0 += chunk_rows) {
+        uint4 t[kMoveVecs];
+        int src[kMoveVecs];
+#pragma unroll
+        for (int i = 0; i < kMoveVecs; ++i) {
+            const int r = r0 + i * rows_per_pass + my_row;
+            src[i] = -1;
+            if (r < keep && my_row < rows_per_pass) {
+                const int s = ix[r];
+                if (s < r || s >= N) set_status(status, kStatusBounds);
+                else if (s != r) src[i] = s;
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < kMoveVecs; ++i)
+            if (src[i] >= 0) t[i] = base[(size_t)src[i] * row_vecs + my_vec];
+        __syncthreads();
+#pragma unroll
+        for (int i = 0; i < kMoveVecs; ++i) {
+            const int r = r0 + i * rows_per_pass + my_row;
+            if (src[i] >= 0) base[(size_t)r * row_vecs + my_vec] = t[i];
+        }
+    }
+}
+
+}  // namespace ipotk
