@@ -1,0 +1,226 @@
+"""GPU parity: the CUDA path through the C ABI against the CPU checker, element by
+element, on seeded inputs (see tests/parity.py for the tolerances)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2410_01518_b200 import inputs, ipot
+from parity import compare_cycle, from_dev_bits, gpu_cycle, make_pot, read_results, to_dev
+
+pytestmark = pytest.mark.gpu
+
+SCORERS = [ipot.IPOT_SCORER_SIMT]
+
+
+def test_config1_tiny_f32_all_units():
+    cfg = inputs.CONFIGS[1]
+    t = inputs.make_cycle(cfg)
+    gpu = gpu_cycle(cfg, t, ipot.IPOT_SCORER_SIMT)
+    same, n = compare_cycle(cfg, t, gpu)
+    assert n == cfg.units and same == n
+
+
+def test_config2_mistral_layer_bf16_all_units():
+    cfg = inputs.CONFIGS[2]
+    t = inputs.make_cycle(cfg)
+    gpu = gpu_cycle(cfg, t, ipot.IPOT_SCORER_SIMT)
+    same, n = compare_cycle(cfg, t, gpu)
+    assert n == cfg.units and same >= n - 1  # at most one unit may sit on a tie
+
+
+SMALL = [
+    # several tiles and a ragged tail, odd sizes, degenerate selections
+    dict(pot_size=96, keep=40, nuc_slots=20, cap_rows=5, Hq=4, Hkv=2, d=64, dtype="f32"),
+    dict(pot_size=333, keep=100, nuc_slots=37, cap_rows=7, Hq=6, Hkv=2, d=64, dtype="bf16"),
+    dict(pot_size=1000, keep=999, nuc_slots=1, cap_rows=3, Hq=2, Hkv=2, d=128, dtype="bf16"),
+    dict(pot_size=200, keep=1, nuc_slots=0, cap_rows=1, Hq=2, Hkv=1, d=128, dtype="f32"),
+    dict(pot_size=257, keep=64, nuc_slots=64, cap_rows=9, Hq=8, Hkv=2, d=64, dtype="bf16"),     # NuC only
+    dict(pot_size=130, keep=65, nuc_slots=0, cap_rows=33, Hq=4, Hkv=4, d=40, dtype="bf16"),     # CaP only, G = 1
+    dict(pot_size=2049, keep=1024, nuc_slots=512, cap_rows=16, Hq=8, Hkv=1, d=128, dtype="bf16", layers=2, batch=2),
+    dict(pot_size=64, keep=63, nuc_slots=30, cap_rows=2, Hq=3, Hkv=3, d=256, dtype="f32", layers=3),
+    dict(pot_size=1500, keep=700, nuc_slots=350, cap_rows=1, Hq=1, Hkv=1, d=128, dtype="bf16", batch=3),  # last-token rule
+]
+
+
+@pytest.mark.parametrize("case", range(len(SMALL)))
+@pytest.mark.parametrize("scorer", SCORERS)
+def test_small_random_shapes(case, scorer):
+    cfg = inputs.small_config(cfg_id=200 + case, **SMALL[case])
+    t = inputs.make_cycle(cfg)
+    gpu = gpu_cycle(cfg, t, scorer)
+    same, n = compare_cycle(cfg, t, gpu)
+    assert n == cfg.units and same >= n - 1
+
+
+def test_partially_filled_pot():
+    cfg = inputs.small_config(cfg_id=220, pot_size=700, keep=300, nuc_slots=100, cap_rows=6, Hq=4, Hkv=2,
+                              d=128, dtype="bf16", layers=2)
+    t = inputs.make_cycle(cfg)
+    gpu = gpu_cycle(cfg, t, n=555)
+    same, n = compare_cycle(cfg, t, gpu, n=555)
+    assert same >= n - 1
+
+
+def test_exact_ties_resolve_to_lower_slots():
+    # all keys identical -> every score equal; all aux equal -> first T slots reserved
+    cfg = inputs.small_config(cfg_id=230, pot_size=300, keep=120, nuc_slots=50, cap_rows=4, d=64, dtype="f32")
+    t = inputs.make_cycle(cfg)
+    t["K"][:] = t["K"][:, :, :, :1, :]
+    t["aux"][:] = 0.25
+    u, idx, K, V = gpu_cycle(cfg, t)
+    for unit in range(cfg.units):
+        assert idx[unit].tolist() == list(range(120))
+        assert np.unique(u[unit]).size == 1
+    same, n = compare_cycle(cfg, t, (u, idx, K, V))
+    assert same == n
+
+
+def test_duplicated_tokens_and_heavy_tails():
+    cfg = inputs.small_config(cfg_id=5, recipe="student_dup", dtype="bf16", pot_size=1200, keep=300,
+                              nuc_slots=150, cap_rows=8, batch=2, Hq=8, Hkv=2, d=128)
+    t = inputs.make_cycle(cfg)
+    gpu = gpu_cycle(cfg, t)
+    compare_cycle(cfg, t, gpu)  # duplicates may swap inside the tie band; bytes must still match
+
+
+def test_outlier_channels_and_lognormal_norms():
+    for recipe, cid in (("stream", 3), ("lognorm", 4)):
+        cfg = inputs.small_config(cfg_id=cid, recipe=recipe, dtype="bf16", pot_size=900, keep=450,
+                                  nuc_slots=225, cap_rows=8, batch=2, Hq=8, Hkv=2, d=128, chunk=900)
+        t = inputs.make_cycle(cfg)
+        same, n = compare_cycle(cfg, t, gpu_cycle(cfg, t))
+        assert same >= n - 1
+
+
+def test_nuc_only_keeps_identical_slots_in_every_head():
+    cfg = inputs.small_config(cfg_id=240, pot_size=500, keep=200, nuc_slots=200, cap_rows=4, Hq=8, Hkv=4,
+                              d=64, dtype="bf16", layers=2)
+    t = inputs.make_cycle(cfg)
+    u, idx, K, V = gpu_cycle(cfg, t)
+    assert (idx == idx[0]).all()
+    assert idx[0].tolist() == oracle.nuc_top(t["aux"][0], 200).tolist()
+
+
+def test_stream_of_cycles_follows_the_checker():
+    """Several fill/distil rounds (Sec. 3.2).  The checker keeps its own pot; after
+    each cycle the GPU's index lists are validated against the checker's scores and
+    the checker's pot is advanced with the validated lists, so a tie resolved the
+    other way does not end the comparison."""
+    cfg = inputs.small_config(cfg_id=3, recipe="stream", dtype="bf16", pot_size=512, keep=256, nuc_slots=128,
+                              cap_rows=8, Hq=8, Hkv=2, d=128, layers=3, chunk=256)
+    h = make_pot(cfg)
+    try:
+        K0, V0 = inputs.make_kv(cfg, 256, chunk=0)
+        ipot.ipot_append_chunk(h, to_dev(K0, "bf16"), to_dev(V0, "bf16"), 256)
+        refK, refV = K0, V0
+        for cyc in range(1, 7):
+            Kc, Vc = inputs.make_kv(cfg, 256, chunk=cyc)
+            ipot.ipot_append_chunk(h, to_dev(Kc, "bf16"), to_dev(Vc, "bf16"), 256)
+            refK, refV = np.concatenate([refK, Kc], axis=3), np.concatenate([refV, Vc], axis=3)
+            t = {"K": refK, "V": refV, "Q": inputs.make_q(cfg, cyc), "aux": inputs.make_aux(cfg, cyc)}
+            ipot.ipot_score_and_compress(h, to_dev(t["Q"], "bf16"), cfg.cap_rows, torch.from_numpy(t["aux"]).cuda())
+            u, idx, K, V = read_results(h, cfg, 512)
+            compare_cycle(cfg, t, (u, idx, K, V))
+            # advance the checker's pot with the validated index lists
+            flatK, flatV = refK.reshape(cfg.units, 512, cfg.d), refV.reshape(cfg.units, 512, cfg.d)
+            refK = np.stack([oracle.gather(flatK[i], idx[i]) for i in range(cfg.units)]).reshape(
+                cfg.layers, cfg.batch, cfg.Hkv, 256, cfg.d)
+            refV = np.stack([oracle.gather(flatV[i], idx[i]) for i in range(cfg.units)]).reshape(
+                cfg.layers, cfg.batch, cfg.Hkv, 256, cfg.d)
+            assert (K.reshape(refK.shape) == refK).all() and (V.reshape(refV.shape) == refV).all()
+    finally:
+        ipot.ipot_destroy(h)
+
+
+def test_host_buffer_calls_match_device_calls():
+    cfg = inputs.small_config(cfg_id=250, pot_size=640, keep=320, nuc_slots=160, cap_rows=8, Hq=8, Hkv=2,
+                              d=128, dtype="bf16", layers=2, batch=2)
+    t = inputs.make_cycle(cfg)
+    dev = gpu_cycle(cfg, t)
+    h = make_pot(cfg)
+    try:
+        ipot.ipot_append_chunk_host(h, t["K"][:, :, :, :400].copy(), t["V"][:, :, :, :400].copy(), 400)
+        ipot.ipot_append_chunk_host(h, t["K"][:, :, :, 400:].copy(), t["V"][:, :, :, 400:].copy(), 240)
+        idx_host = np.full((cfg.units, cfg.keep), -1, dtype=np.int32)
+        ipot.ipot_score_and_compress_host(h, t["Q"], cfg.cap_rows, t["aux"], idx_host)
+        u, idx, K, V = read_results(h, cfg, 640)
+        assert (idx_host == idx).all()
+        assert (idx == dev[1]).all() and (K == dev[2]).all() and (V == dev[3]).all() and (u == dev[0]).all()
+    finally:
+        ipot.ipot_destroy(h)
+
+
+def test_state_machine_and_argument_errors():
+    cfg = inputs.small_config(cfg_id=260, pot_size=128, keep=64, nuc_slots=32, cap_rows=4, d=64, dtype="bf16")
+    t = inputs.make_cycle(cfg)
+    h = make_pot(cfg)
+    L = ipot.lib()
+    try:
+        Kd, Vd, Qd = to_dev(t["K"], "bf16"), to_dev(t["V"], "bf16"), to_dev(t["Q"], "bf16")
+        auxd = torch.from_numpy(t["aux"]).cuda()
+        assert L.ipot_score_and_compress(h, Qd.data_ptr(), 4, auxd.data_ptr()) == ipot.IPOT_E_STATE  # empty
+        ipot.ipot_append_chunk(h, Kd[:, :, :, :64].contiguous(), Vd[:, :, :, :64].contiguous(), 64)
+        assert L.ipot_score_and_compress(h, Qd.data_ptr(), 4, auxd.data_ptr()) == ipot.IPOT_E_STATE  # len == keep
+        assert L.ipot_append_chunk(h, Kd.data_ptr(), Vd.data_ptr(), 65) == ipot.IPOT_E_STATE          # overflow
+        assert ipot.ipot_view(h)[2] == 64
+        assert L.ipot_append_chunk(h, Kd.data_ptr() + 2, Vd.data_ptr(), 1) == ipot.IPOT_E_INVALID     # misaligned
+        assert L.ipot_append_chunk(h, Kd.data_ptr(), Vd.data_ptr(), 0) == ipot.IPOT_E_INVALID
+        ipot.ipot_append_chunk(h, Kd[:, :, :, 64:].contiguous(), Vd[:, :, :, 64:].contiguous(), 64)
+        assert L.ipot_score_and_compress(h, Qd.data_ptr(), 5, auxd.data_ptr()) == ipot.IPOT_E_INVALID  # > max rows
+        assert L.ipot_score_and_compress(h, Qd.data_ptr(), 4, None) == ipot.IPOT_E_INVALID             # T > 0, no aux
+        assert L.ipot_set_nuc_slots(h, 65) == ipot.IPOT_E_INVALID
+        assert L.ipot_set_scorer(h, 7) == ipot.IPOT_E_INVALID
+        assert ipot.ipot_view(h)[2] == 128
+        ipot.ipot_score_and_compress(h, Qd, 4, auxd)
+        assert ipot.ipot_view(h)[2] == 64 and ipot.ipot_sync_status(h) == 0
+        ipot.ipot_reset(h)
+        assert ipot.ipot_view(h)[2] == 0
+        assert ipot.ipot_launch_count(h) >= 6
+    finally:
+        ipot.ipot_destroy(h)
+
+
+def test_set_nuc_slots_and_profiling_and_determinism():
+    cfg = inputs.small_config(cfg_id=270, pot_size=777, keep=300, nuc_slots=0, cap_rows=8, Hq=8, Hkv=2, d=128,
+                              dtype="bf16", layers=2)
+    t = inputs.make_cycle(cfg)
+    a = gpu_cycle(cfg, t)
+    b = gpu_cycle(cfg, t)
+    for x, y in zip(a, b):
+        assert (x == y).all()  # same bytes twice
+    h = make_pot(cfg, nuc_slots=10)
+    try:
+        ipot.ipot_set_nuc_slots(h, 0)
+        ipot.ipot_set_profiling(h, 1)
+        ipot.ipot_append_chunk(h, to_dev(t["K"], "bf16"), to_dev(t["V"], "bf16"), 777)
+        ipot.ipot_score_and_compress(h, to_dev(t["Q"], "bf16"), 8, None)
+        ms, scorer = ipot.ipot_last_kernel_ms(h)
+        assert len(ms) == 4 and all(m >= 0 for m in ms) and ms[1] > 0 and scorer in (1, 2)
+        c = read_results(h, cfg, 777)
+        assert (c[1] == a[1]).all()
+    finally:
+        ipot.ipot_destroy(h)
+
+
+def test_score_only_leaves_the_pot_alone():
+    cfg = inputs.small_config(cfg_id=280, pot_size=400, keep=100, nuc_slots=50, cap_rows=8, Hq=8, Hkv=2, d=128,
+                              dtype="bf16")
+    t = inputs.make_cycle(cfg)
+    h = make_pot(cfg)
+    try:
+        Kd, Vd = to_dev(t["K"], "bf16"), to_dev(t["V"], "bf16")
+        ipot.ipot_append_chunk(h, Kd, Vd, 400)
+        ipot.ipot_score_only(h, to_dev(t["Q"], "bf16"), 8)
+        assert ipot.ipot_sync_status(h) == 0
+        sp, nb = ipot.ipot_last_scores(h)
+        u = ipot.device_array(sp, (cfg.units, nb), "f32").cpu().numpy()
+        Kp, Vp, ln = ipot.ipot_view(h)
+        assert ln == 400 and nb == 400
+        assert (from_dev_bits(ipot.device_array(Kp, (cfg.units, 400, 128), "bf16"), "bf16")
+                == t["K"].reshape(cfg.units, 400, 128)).all()
+        ref = oracle.cycle(t["Q"], t["K"], t["V"], t["aux"], cfg.keep, cfg.nuc_slots, with_kv=False)
+        np.testing.assert_allclose(u, ref["u"], rtol=1e-3, atol=1e-30)
+        assert abs(u.sum(axis=1) - cfg.G * cfg.cap_rows).max() < 1e-2
+    finally:
+        ipot.ipot_destroy(h)
