@@ -1,0 +1,332 @@
+#!/usr/bin/env python
+"""Benchmark of the CCD compression cycle (one JSON line on stdout).
+
+A step is one pass of the whole hot path over one batch of synthetic input:
+append a chunk of new K/V rows behind the survivors, then one
+``ipot_score_and_compress`` (NuC ranking, CaP scoring, per-head selection, in-place
+K/V compaction) over all layers x streams x kv-heads.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg3|cfg2|cfg4|cfg5]
+    python bench.py --impl reference ...      # the CPU checker, as it stands, on the host cores
+
+With N > 1 (under torchrun) every rank runs an independent replica on its own GPU:
+the cycle has no exchange step, so there is no collective on the data path.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2410_01518_b200 import inputs  # noqa: E402
+
+WORKLOADS = {"cfg2": 2, "cfg3": 3, "cfg4": 4, "cfg5": 5}
+RING = 4  # distinct chunks / query sets cycled through
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1400.0, "source": "fallback"}
+
+
+def workload_shape(cfg):
+    """(rows appended per step, rows in the pot when the cycle runs)."""
+    n_new = cfg.pot_size - cfg.keep
+    return n_new, cfg.pot_size
+
+
+def gen_ring(cfg, n_new):
+    """RING chunks of new K/V rows, CaP queries and novelty scores (numpy, storage dtype)."""
+    ring = []
+    for i in range(RING):
+        K, V = inputs.make_kv(cfg, n_new, chunk=1 + i)
+        ring.append({"K": K, "V": V, "Q": inputs.make_q(cfg, 1 + i), "aux": inputs.make_aux(cfg, 1 + i)})
+    K0, V0 = inputs.make_kv(cfg, cfg.keep, chunk=0)
+    return ring, K0, V0
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle samples taken while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+
+    def start(self):
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                       "--format=csv,noheader,nounits", "-lms", "50"], stdout=self.f,
+                                      stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        rows = [r.split(",") for r in open(self.f.name).read().strip().splitlines() if r.count(",") >= 8]
+        os.unlink(self.f.name)
+        sm, reasons = [], set()
+        for r in rows:
+            r = [x.strip() for x in r]
+            try:
+                sm.append(float(r[1]))
+                out["sm_max_mhz"] = float(r[2])
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if sm:
+            out["sm_mhz"] = float(np.median(sm))
+            out["samples"] = len(sm)
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+def cpu_baseline(cfg, ring, K0, V0, n_units_sample, threads=None):
+    """The checker, as it stands, on a sample of the units of one cycle."""
+    import oracle
+    if threads:
+        oracle.set_threads(threads)
+    t = ring[0]
+    K = np.concatenate([K0, t["K"]], axis=3)
+    V = np.concatenate([V0, t["V"]], axis=3)
+    units = np.linspace(0, cfg.units - 1, n_units_sample).astype(np.int32)
+    oracle.cycle(t["Q"], K, V, t["aux"], cfg.keep, cfg.nuc_slots, units=units[:1])  # load the library
+    t0 = time.perf_counter()
+    oracle.cycle(t["Q"], K, V, t["aux"], cfg.keep, cfg.nuc_slots, units=units)
+    dt = time.perf_counter() - t0
+    cycles_per_s = (len(units) / cfg.units) / dt
+    return cycles_per_s, dt, len(units), oracle.max_threads()
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    n_new, N = workload_shape(cfg)
+    small = cfg.with_layers(min(cfg.layers, 2))  # the sample only needs a few layers' tensors
+    ring, K0, V0 = gen_ring(small, n_new)
+    n_sample = min(small.units, 16)
+    for _ in range(args.warmup):
+        cpu_baseline(small, ring, K0, V0, 1)
+    times = []
+    for _ in range(args.steps):
+        _, dt, n_units, threads = cpu_baseline(small, ring, K0, V0, n_sample)
+        times.append(dt)
+    ms = float(np.mean(times)) * 1e3 * cfg.units / n_sample  # one full cycle, extrapolated
+    value = 1e3 / ms
+    line = {
+        "impl": "reference", "metric": "ccd_cycles_per_s", "value": value, "unit": "cycles/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": config_dict(cfg, n_new, N),
+        "cpu_baseline": {"value": value, "unit": "cycles/s", "cores": threads, "kind": "oracle",
+                         "sample": f"{n_sample} of {cfg.units} units of one cycle per step (units are independent and "
+                                   f"equal-sized); full-cycle time extrapolated"},
+        "e2e": {"value": value, "unit": "cycles/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "pot_tokens_per_s": value * N * cfg.batch,
+    }
+    print(json.dumps(line))
+
+
+def config_dict(cfg, n_new, N):
+    return {"workload": f"configs[{cfg.cfg_id - 1}] {cfg.name}: one CCD cycle per step "
+                        f"(append {n_new} rows, distil {N} -> {cfg.keep})",
+            "layers": cfg.layers, "batch": cfg.batch, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "d": cfg.d,
+            "pot_size": cfg.pot_size, "keep": cfg.keep, "nuc_slots": cfg.nuc_slots, "cap_rows": cfg.cap_rows,
+            "units": cfg.units, "l2": "inputs_larger_than_l2" if cfg.units * N * cfg.d * cfg.elem_bytes * 2 > 126e6
+            else "l2_flushed_between_steps"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg3", choices=sorted(WORKLOADS))
+    ap.add_argument("--scorer", default="auto", choices=["auto", "simt", "tensor"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    cfg = inputs.CONFIGS[WORKLOADS[args.workload]]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2410_01518_b200 import ipot
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the compression path has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    n_new, N = workload_shape(cfg)
+    ring, K0, V0 = gen_ring(cfg, n_new)
+    tdt = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
+
+    def dev(a):
+        t = torch.from_numpy(a.view(np.int16) if cfg.dtype == "bf16" and a.dtype == np.uint16 else a).cuda()
+        return t.view(tdt) if a.dtype == np.uint16 else t
+
+    def pin(a):
+        return torch.from_numpy(a.view(np.int16) if a.dtype == np.uint16 else a).pin_memory()
+
+    dring = [{k: dev(v) for k, v in t.items()} for t in ring]
+    hring = [{k: pin(v) for k, v in t.items()} for t in ring]
+    K0d, V0d = dev(K0), dev(V0)
+    idx_host = torch.empty((cfg.units, cfg.keep), dtype=torch.int32).pin_memory()
+
+    h = ipot.ipot_create_ex(cfg.pot_size, cfg.keep, cfg.layers, cfg.Hq, cfg.Hkv, cfg.d, batch=cfg.batch,
+                            dtype=ipot.IPOT_BF16 if cfg.dtype == "bf16" else ipot.IPOT_F32,
+                            nuc_slots=cfg.nuc_slots, max_cap_rows=cfg.cap_rows)
+    ipot.ipot_set_scorer(h, {"auto": 0, "simt": 1, "tensor": 2}[args.scorer])
+    stream = torch.cuda.current_stream()
+    ipot.ipot_set_stream(h, stream.cuda_stream)
+    ipot.ipot_append_chunk(h, K0d, V0d, cfg.keep)
+
+    small_l2 = cfg.units * N * cfg.d * cfg.elem_bytes * 2 <= 126e6
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda") if small_l2 else None
+
+    def step_dev(i):
+        t = dring[i % RING]
+        if flush is not None:
+            flush.add_(1)
+        ipot.ipot_append_chunk(h, t["K"], t["V"], n_new)
+        ipot.ipot_score_and_compress(h, t["Q"], cfg.cap_rows, t["aux"])
+
+    def step_host(i):
+        t = hring[i % RING]
+        ipot.ipot_append_chunk_host(h, t["K"], t["V"], n_new)
+        ipot.ipot_score_and_compress_host(h, t["Q"], cfg.cap_rows, t["aux"], idx_host)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(step, steps, warmup, sampler=None):
+        for i in range(warmup):
+            step(i)
+        barrier()
+        if sampler:
+            sampler.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        l0 = ipot.ipot_launch_count(h)
+        e0.record(stream)
+        for i in range(steps):
+            step(warmup + i)
+        e1.record(stream)
+        barrier()
+        clocks = sampler.stop() if sampler else None
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            tt = torch.tensor([ms], device="cuda")
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            ms = float(tt.item())
+        return ms, ipot.ipot_launch_count(h) - l0, clocks
+
+    # device-resident inputs: the headline value, with per-kernel events over the same timed region
+    ipot.ipot_set_profiling(h, 1)
+    for i in range(args.warmup):
+        step_dev(i)
+    torch.cuda.synchronize()
+    ipot.ipot_kernel_ms(h)  # drop the warm-up cycles from the per-kernel means
+    sampler = ClockSampler(local)
+    ms_total, launches, clocks = timed(step_dev, args.steps, 0, sampler)
+    kms, kcycles, scorer_used = ipot.ipot_kernel_ms(h)
+    ipot.ipot_set_profiling(h, 0)
+    assert ipot.ipot_sync_status(h) == 0, "device status is not clean"
+    ms_step = ms_total / args.steps
+    value = world * 1e3 / ms_step
+
+    # end to end: host (pinned) buffers in, index lists out, copies inside the timed region
+    e2e_steps = max(3, min(args.steps, 50))
+    ms_e2e, _, _ = timed(step_host, e2e_steps, 3)
+    assert ipot.ipot_sync_status(h) == 0
+    e2e_value = world * 1e3 / (ms_e2e / e2e_steps)
+    h2d = sum(hring[0][k].numel() * hring[0][k].element_size() for k in ("K", "V", "Q", "aux"))
+    d2h = idx_host.numel() * 4
+
+    # roofline of the dominant kernel
+    pk = peaks()
+    units, e, d, M = cfg.units, cfg.elem_bytes, cfg.d, cfg.G * cfg.cap_rows
+    score_bytes = units * (N * d * e + M * d * e + 4 * N)      # K once + Q + scores out
+    score_flops = 2.0 * units * M * N * d
+    compact_bytes = units * 4 * cfg.keep * d * e                # K and V, read + write, all kept rows
+    names = ["nuc_rank", "cap_score", "select", "compact"]
+    dom = int(np.argmax(kms))
+    if names[dom] == "compact":
+        roof = {"kernel": "compact_kernel", "bound": "hbm", "achieved": compact_bytes / (kms[3] * 1e-3) / 1e9,
+                "peak": pk["hbm_gbs"], "unit": "GB/s"}
+    else:
+        roof = {"kernel": "cap_score (" + ("tcgen05" if scorer_used == 2 else "simt") + ")", "bound": "hbm",
+                "achieved": score_bytes / (kms[1] * 1e-3) / 1e9, "peak": pk["hbm_gbs"], "unit": "GB/s"}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["peak_source"] = pk["source"]
+    roof["traffic"] = None
+    roof["kernel_ms"] = dict(zip(names, [round(x, 5) for x in kms]))
+    roof["cycles_averaged"] = kcycles
+    roof["cap_score_gbs"] = score_bytes / (kms[1] * 1e-3) / 1e9
+    roof["cap_score_tflops"] = score_flops / (kms[1] * 1e-3) / 1e12
+    roof["compact_gbs"] = compact_bytes / (kms[3] * 1e-3) / 1e9
+
+    line = {
+        "metric": "ccd_cycles_per_s", "value": value, "unit": "cycles/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
+        "config": config_dict(cfg, n_new, N),
+        "pot_tokens_per_s": value * N * cfg.batch,
+        "layer_cycles_per_s": value * cfg.layers,
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": "cycles/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "steps": e2e_steps},
+        "gpu_launches": launches,
+        "roofline": roof,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        n_sample = max(8, min(cfg.units, 64))
+        v, dt, n_units, threads = cpu_baseline(cfg, ring, K0, V0, n_sample)
+        line["cpu_baseline"] = {"value": v, "unit": "cycles/s", "cores": threads, "kind": "oracle",
+                                "sample": f"{n_units} of {cfg.units} units of one cycle in {dt:.1f} s; "
+                                          f"full-cycle rate extrapolated (units are independent and equal-sized)"}
+    ipot.ipot_destroy(h)
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

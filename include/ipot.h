@@ -161,14 +161,16 @@ int ipot_last_scores(ipot_t *pot, const float **u, int *len_before); /* [layers]
 int ipot_sync_status(ipot_t *pot);
 
 /*
- * Per-kernel device timing.  When enabled, every cycle records CUDA events on
- * the pot's stream around its kernels; ipot_last_kernel_ms() waits for the last
- * cycle and returns, in milliseconds: ms[0] NuC ranking, ms[1] CaP scoring,
- * ms[2] per-head selection, ms[3] K/V compaction.  *scorer_used (may be NULL)
- * receives IPOT_SCORER_SIMT or IPOT_SCORER_TENSOR.
+ * Per-kernel device timing.  While enabled, every cycle (up to 512 between
+ * reads) records CUDA events on the pot's stream around its kernels; nothing
+ * waits.  ipot_kernel_ms() waits for the last recorded cycle, returns the MEAN
+ * over the recorded cycles in milliseconds - ms[0] NuC ranking, ms[1] CaP
+ * scoring, ms[2] per-head selection, ms[3] K/V compaction - and starts a new
+ * series.  *cycles (may be NULL) = cycles averaged; *scorer_used (may be NULL)
+ * = IPOT_SCORER_SIMT or IPOT_SCORER_TENSOR.  STATE if nothing was recorded.
  */
 int ipot_set_profiling(ipot_t *pot, int on);
-int ipot_last_kernel_ms(ipot_t *pot, float ms[4], int *scorer_used);
+int ipot_kernel_ms(ipot_t *pot, float ms[4], int *cycles, int *scorer_used);
 
 /* Number of kernels this pot has launched since it was created. */
 int ipot_launch_count(ipot_t *pot, long long *launches);

@@ -42,13 +42,15 @@ struct ipot {
     int last_scorer;
     // timing
     int profiling;
-    cudaEvent_t ev[5];
-    bool ev_valid;
+    cudaEvent_t (*ev)[5];  // kProfSlots event quintuples, one per recorded cycle
+    int ev_used;
     long long launches;
     TcPlan tc;           // tensor-core scorer state
 };
 
 namespace {
+
+constexpr int kProfSlots = 512;
 
 #define IPOT_CUDA(call)                                                             \
     do {                                                                            \
@@ -80,7 +82,11 @@ void free_all(ipot *p)
     cudaFree(p->K); cudaFree(p->V); cudaFree(p->scores); cudaFree(p->summed);
     cudaFree(p->row_stats); cudaFree(p->nuc_mask); cudaFree(p->idx); cudaFree(p->status);
     cudaFree(p->stage_q); cudaFree(p->stage_aux);
-    for (auto &e : p->ev) if (e) cudaEventDestroy(e);
+    if (p->ev) {
+        for (int i = 0; i < kProfSlots; ++i)
+            for (auto &e : p->ev[i]) if (e) cudaEventDestroy(e);
+        delete[] p->ev;
+    }
 }
 
 template <typename T>
@@ -110,14 +116,15 @@ int run_scoring(ipot *p, const void *Q, int cap_rows, const float *aux, int *par
     if (scorer == IPOT_SCORER_TENSOR && !tc_ok) return IPOT_E_INVALID;
     if (scorer == IPOT_SCORER_AUTO) scorer = tc_ok ? IPOT_SCORER_TENSOR : IPOT_SCORER_SIMT;
 
-    if (p->profiling) IPOT_CUDA(cudaEventRecord(p->ev[0], p->stream));
+    cudaEvent_t *ev = (p->profiling && p->ev_used < kProfSlots) ? p->ev[p->ev_used] : nullptr;
+    if (ev) IPOT_CUDA(cudaEventRecord(ev[0], p->stream));
     if (T > 0 && aux) {
         IPOT_CUDA(cudaFuncSetAttribute(nuc_mask_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 32768 * 4));
         nuc_mask_kernel<<<p->cfg.batch, kSelThreads, (size_t)N * 4, p->stream>>>(aux, p->nuc_mask, N, T);
         p->launches += 1;
         IPOT_CUDA(cudaGetLastError());
     }
-    if (p->profiling) IPOT_CUDA(cudaEventRecord(p->ev[1], p->stream));
+    if (ev) IPOT_CUDA(cudaEventRecord(ev[1], p->stream));
     *parts = 1;
     int rc;
     if (scorer == IPOT_SCORER_TENSOR) {
@@ -129,7 +136,7 @@ int run_scoring(ipot *p, const void *Q, int cap_rows, const float *aux, int *par
         rc = p->cfg.dtype == IPOT_F32 ? launch_simt<float>(p, Q, M, N) : launch_simt<__nv_bfloat16>(p, Q, M, N);
     }
     if (rc != IPOT_OK) return rc;
-    if (p->profiling) IPOT_CUDA(cudaEventRecord(p->ev[2], p->stream));
+    if (ev) IPOT_CUDA(cudaEventRecord(ev[2], p->stream));
     p->last_scorer = scorer;
     p->last_len_before = N;
     p->last_scores = (*parts > 1) ? p->summed : p->scores;
@@ -162,6 +169,7 @@ int run_cycle(ipot *p, const void *Q, int cap_rows, const float *aux)
 {
     const int N = p->len, keep = p->cfg.keep, T = p->cfg.nuc_slots;
     int parts = 1;
+    cudaEvent_t *ev = (p->profiling && p->ev_used < kProfSlots) ? p->ev[p->ev_used] : nullptr;
     int rc = run_scoring(p, Q, cap_rows, aux, &parts);
     if (rc != IPOT_OK) return rc;
     const size_t part_stride = (size_t)p->units * p->cfg.pot_size;
@@ -171,7 +179,7 @@ int run_cycle(ipot *p, const void *Q, int cap_rows, const float *aux)
         parts > 1 ? p->summed : nullptr, N, keep, p->cfg.Hkv, p->cfg.batch, p->status);
     p->launches += 1;
     IPOT_CUDA(cudaGetLastError());
-    if (p->profiling) IPOT_CUDA(cudaEventRecord(p->ev[3], p->stream));
+    if (ev) IPOT_CUDA(cudaEventRecord(ev[3], p->stream));
 
     const int row_vecs = p->row_bytes / 16;
     const int slices = compact_slices(p);
@@ -180,9 +188,9 @@ int run_cycle(ipot *p, const void *Q, int cap_rows, const float *aux)
                                                         row_vecs / slices, (size_t)p->cfg.pot_size * row_vecs, p->status);
     p->launches += 1;
     IPOT_CUDA(cudaGetLastError());
-    if (p->profiling) {
-        IPOT_CUDA(cudaEventRecord(p->ev[4], p->stream));
-        p->ev_valid = true;
+    if (ev) {
+        IPOT_CUDA(cudaEventRecord(ev[4], p->stream));
+        p->ev_used += 1;
     }
     p->len = keep;
     return IPOT_OK;
@@ -241,8 +249,11 @@ int ipot_create_ex(const ipot_config_t *cfg, ipot_t **out)
     alloc(&p->stage_q, (size_t)p->units * maxM * p->row_bytes);
     alloc((void **)&p->stage_aux, (size_t)cfg->batch * cfg->pot_size * 4);
     if (ok) ok = cudaMemset(p->status, 0, 16) == cudaSuccess;
-    for (auto &e : p->ev)
-        if (ok && cudaEventCreate(&e) != cudaSuccess) ok = false;
+    p->ev = new (std::nothrow) cudaEvent_t[kProfSlots][5]();
+    if (!p->ev) ok = false;
+    for (int i = 0; ok && i < kProfSlots; ++i)
+        for (auto &e : p->ev[i])
+            if (ok && cudaEventCreate(&e) != cudaSuccess) ok = false;
     if (!ok) {
         cudaGetLastError();
         free_all(p);
@@ -397,17 +408,26 @@ int ipot_set_profiling(ipot_t *p, int on)
 {
     if (!p) return IPOT_E_INVALID;
     p->profiling = on != 0;
-    p->ev_valid = false;
+    p->ev_used = 0;
     return IPOT_OK;
 }
 
-int ipot_last_kernel_ms(ipot_t *p, float ms[4], int *scorer_used)
+int ipot_kernel_ms(ipot_t *p, float ms[4], int *cycles, int *scorer_used)
 {
     if (!p || !ms) return IPOT_E_INVALID;
-    if (!p->profiling || !p->ev_valid) return IPOT_E_STATE;
-    IPOT_CUDA(cudaEventSynchronize(p->ev[4]));
-    for (int i = 0; i < 4; ++i) IPOT_CUDA(cudaEventElapsedTime(&ms[i], p->ev[i], p->ev[i + 1]));
+    if (!p->profiling || p->ev_used == 0) return IPOT_E_STATE;
+    IPOT_CUDA(cudaEventSynchronize(p->ev[p->ev_used - 1][4]));
+    double sum[4] = {0, 0, 0, 0};
+    for (int c = 0; c < p->ev_used; ++c)
+        for (int i = 0; i < 4; ++i) {
+            float t = 0.f;
+            IPOT_CUDA(cudaEventElapsedTime(&t, p->ev[c][i], p->ev[c][i + 1]));
+            sum[i] += t;
+        }
+    for (int i = 0; i < 4; ++i) ms[i] = (float)(sum[i] / p->ev_used);
+    if (cycles) *cycles = p->ev_used;
     if (scorer_used) *scorer_used = p->last_scorer;
+    p->ev_used = 0;
     return IPOT_OK;
 }
 

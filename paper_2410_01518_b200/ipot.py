@@ -26,7 +26,7 @@ SYMBOLS = [
     "ipot_set_scorer", "ipot_reset", "ipot_append_chunk", "ipot_append_chunk_host",
     "ipot_score_and_compress", "ipot_score_and_compress_host", "ipot_score_only", "ipot_view",
     "ipot_last_indices", "ipot_last_scores", "ipot_sync_status", "ipot_set_profiling",
-    "ipot_last_kernel_ms", "ipot_launch_count", "ipot_strerror",
+    "ipot_kernel_ms", "ipot_launch_count", "ipot_strerror",
 ]
 
 
@@ -75,7 +75,7 @@ def lib() -> C.CDLL:
         L.ipot_last_scores.argtypes = [vp, C.POINTER(vp), C.POINTER(ip)]
         L.ipot_sync_status.argtypes = [vp]
         L.ipot_set_profiling.argtypes = [vp, ip]
-        L.ipot_last_kernel_ms.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(ip)]
+        L.ipot_kernel_ms.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(ip), C.POINTER(ip)]
         L.ipot_launch_count.argtypes = [vp, C.POINTER(C.c_longlong)]
         L.ipot_strerror.argtypes = [ip]
         L.ipot_strerror.restype = C.c_char_p
@@ -189,12 +189,12 @@ def ipot_set_profiling(h, on) -> None:
     _check(lib().ipot_set_profiling(h, int(on)), "ipot_set_profiling")
 
 
-def ipot_last_kernel_ms(h):
-    """-> ([nuc, score, select, compact] milliseconds, scorer used)."""
+def ipot_kernel_ms(h):
+    """-> ([nuc, score, select, compact] mean milliseconds, cycles averaged, scorer used)."""
     ms = (C.c_float * 4)()
-    s = C.c_int()
-    _check(lib().ipot_last_kernel_ms(h, ms, C.byref(s)), "ipot_last_kernel_ms")
-    return list(ms), s.value
+    n, s = C.c_int(), C.c_int()
+    _check(lib().ipot_kernel_ms(h, ms, C.byref(n), C.byref(s)), "ipot_kernel_ms")
+    return list(ms), n.value, s.value
 
 
 def ipot_launch_count(h) -> int:

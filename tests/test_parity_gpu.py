@@ -195,8 +195,8 @@ def test_set_nuc_slots_and_profiling_and_determinism():
         ipot.ipot_set_profiling(h, 1)
         ipot.ipot_append_chunk(h, to_dev(t["K"], "bf16"), to_dev(t["V"], "bf16"), 777)
         ipot.ipot_score_and_compress(h, to_dev(t["Q"], "bf16"), 8, None)
-        ms, scorer = ipot.ipot_last_kernel_ms(h)
-        assert len(ms) == 4 and all(m >= 0 for m in ms) and ms[1] > 0 and scorer in (1, 2)
+        ms, cycles, scorer = ipot.ipot_kernel_ms(h)
+        assert cycles == 1 and len(ms) == 4 and all(m >= 0 for m in ms) and ms[1] > 0 and scorer in (1, 2)
         c = read_results(h, cfg, 777)
         assert (c[1] == a[1]).all()
     finally:
