@@ -166,7 +166,7 @@ def config_dict(cfg, n_new, N):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg3", choices=sorted(WORKLOADS))
@@ -316,7 +316,7 @@ def main():
         "roofline": roof,
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        n_sample = max(8, min(cfg.units, 64))
+        n_sample = min(cfg.units, 256)
         v, dt, n_units, threads = cpu_baseline(cfg, ring, K0, V0, n_sample)
         line["cpu_baseline"] = {"value": v, "unit": "cycles/s", "cores": threads, "kind": "oracle",
                                 "sample": f"{n_units} of {cfg.units} units of one cycle in {dt:.1f} s; "

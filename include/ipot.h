@@ -161,7 +161,7 @@ int ipot_last_scores(ipot_t *pot, const float **u, int *len_before); /* [layers]
 int ipot_sync_status(ipot_t *pot);
 
 /*
- * Per-kernel device timing.  While enabled, every cycle (up to 512 between
+ * Per-kernel device timing.  While enabled, every cycle (up to 2048 between
  * reads) records CUDA events on the pot's stream around its kernels; nothing
  * waits.  ipot_kernel_ms() waits for the last recorded cycle, returns the MEAN
  * over the recorded cycles in milliseconds - ms[0] NuC ranking, ms[1] CaP

@@ -50,7 +50,7 @@ struct ipot {
 
 namespace {
 
-constexpr int kProfSlots = 512;
+constexpr int kProfSlots = 2048;
 
 #define IPOT_CUDA(call)                                                             \
     do {                                                                            \
@@ -249,11 +249,6 @@ int ipot_create_ex(const ipot_config_t *cfg, ipot_t **out)
     alloc(&p->stage_q, (size_t)p->units * maxM * p->row_bytes);
     alloc((void **)&p->stage_aux, (size_t)cfg->batch * cfg->pot_size * 4);
     if (ok) ok = cudaMemset(p->status, 0, 16) == cudaSuccess;
-    p->ev = new (std::nothrow) cudaEvent_t[kProfSlots][5]();
-    if (!p->ev) ok = false;
-    for (int i = 0; ok && i < kProfSlots; ++i)
-        for (auto &e : p->ev[i])
-            if (ok && cudaEventCreate(&e) != cudaSuccess) ok = false;
     if (!ok) {
         cudaGetLastError();
         free_all(p);
@@ -407,6 +402,12 @@ int ipot_sync_status(ipot_t *p)
 int ipot_set_profiling(ipot_t *p, int on)
 {
     if (!p) return IPOT_E_INVALID;
+    if (on && !p->ev) {  // the event pool is created on first use
+        p->ev = new (std::nothrow) cudaEvent_t[kProfSlots][5]();
+        if (!p->ev) return IPOT_E_NOMEM;
+        for (int i = 0; i < kProfSlots; ++i)
+            for (auto &e : p->ev[i]) IPOT_CUDA(cudaEventCreate(&e));
+    }
     p->profiling = on != 0;
     p->ev_used = 0;
     return IPOT_OK;
