@@ -51,7 +51,8 @@ enum {
     IPOT_E_NOMEM = -3,   /* device or host allocation failed */
     IPOT_E_CUDA = -4,    /* a CUDA runtime/driver call failed, or no device */
     IPOT_E_TIMEOUT = -5, /* a bounded device-side wait gave up (sticky, reported by ipot_sync_status) */
-    IPOT_E_BOUNDS = -6   /* a device-side self-check found an index out of range (sticky) */
+    IPOT_E_BOUNDS = -6,  /* a device-side self-check found an index out of range (sticky) */
+    IPOT_E_LIMIT = -7    /* a size exceeds the fixed scratch of ipot_cap_scores_noalloc() */
 };
 
 enum { IPOT_BF16 = 0, IPOT_F32 = 1 };
@@ -176,6 +177,43 @@ int ipot_kernel_ms(ipot_t *pot, float ms[4], int *cycles, int *scorer_used);
 int ipot_launch_count(ipot_t *pot, long long *launches);
 
 const char *ipot_strerror(int code);
+
+/*
+ * CaP scoring for callers that must not allocate device memory.  (The paper has
+ * no counterpart: this is a packaging variant of the scoring step, computing the
+ * same u_j as step 2 of ipot_score_and_compress() with the fp32 FMA kernels.)
+ *
+ * Who needs it: processes whose device memory is handed over, whole, to a
+ * framework's own pool at start-up, where a later cudaMalloc can fail or eat
+ * into that pool's reserve; and latency-sensitive loops, because cudaMalloc
+ * and cudaFree synchronise the whole device and so stall every other stream.
+ * No pot object is involved.  This call makes no cudaMalloc/cudaFree and calls
+ * no allocating routine; its only scratch - one (max, 1/denominator) pair per
+ * query row, handed from its first kernel launch to its second - is a fixed
+ * array of IPOT_NOALLOC_MAX_ROWS pairs (512 KiB) that is part of the library
+ * image, so every device that loads the library carries it until the process
+ * exits.
+ *
+ *   Q       device [units][rows][d]          query rows of each unit (rows = G * cap_rows)
+ *   K       device [units][k_unit_rows][d]   keys; the first N rows of each unit are scored
+ *   scores  device [units][N] f32            output, fully overwritten
+ *   dtype   IPOT_BF16 or IPOT_F32 (element type of Q and K); d as for ipot_create()
+ *   cuda_stream  cudaStream_t (NULL = default stream); the call only queues work
+ *
+ * Limits and errors: units * rows > IPOT_NOALLOC_MAX_ROWS -> IPOT_E_LIMIT,
+ * nothing is launched.  INVALID for NULL/misaligned pointers or bad sizes, CUDA
+ * for runtime failures.
+ * First use on a device: the first call made while a given device is current
+ * looks up the array's device address (cudaGetSymbolAddress) and keeps it; make
+ * that first call outside any stream capture.
+ * Sharing: all calls on a device use the same array, and it keeps whatever the
+ * last call left there.  Nothing has to be cleared, because each call writes
+ * every entry it later reads; but two calls whose kernels can overlap on the
+ * GPU (different streams, no ordering between them) race on it - order them.
+ */
+#define IPOT_NOALLOC_MAX_ROWS 65536
+int ipot_cap_scores_noalloc(const void *Q, const void *K, float *scores, int units, int rows, int N, int d,
+                            int k_unit_rows, int dtype, void *cuda_stream);
 
 #ifdef __cplusplus
 }

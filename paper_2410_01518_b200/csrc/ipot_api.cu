@@ -6,6 +6,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "common.cuh"
@@ -449,8 +450,72 @@ const char *ipot_strerror(int code)
     case IPOT_E_CUDA: return "CUDA call failed or no usable device";
     case IPOT_E_TIMEOUT: return "a bounded device-side wait gave up";
     case IPOT_E_BOUNDS: return "a device-side self-check found an index out of range";
+    case IPOT_E_LIMIT: return "size exceeds the fixed scratch capacity of the allocation-free entry point";
     default: return "unknown error code";
     }
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------
+// Allocation-free CaP scoring.  The two SIMT launches hand the per-row softmax
+// statistics to each other through global memory; here that scratch is a fixed
+// array inside the library image instead of a cudaMalloc'ed buffer.
+// ---------------------------------------------------------------------------
+static __device__ __align__(256) float2 g_noalloc_row_stats[IPOT_NOALLOC_MAX_ROWS];
+
+namespace {
+std::mutex g_noalloc_mutex;
+float2 *g_noalloc_ptr[64];  // device address of the array, per device ordinal
+
+// The array's name is only a host-side handle; kernels need the address the
+// runtime reports for the device that is current.
+int noalloc_scratch(float2 **out)
+{
+    int dev = 0;
+    IPOT_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return IPOT_E_INVALID;
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!g_noalloc_ptr[dev]) {
+        void *ptr = nullptr;
+        IPOT_CUDA(cudaGetSymbolAddress(&ptr, g_noalloc_row_stats));
+        g_noalloc_ptr[dev] = static_cast<float2 *>(ptr);
+    }
+    *out = g_noalloc_ptr[dev];
+    return IPOT_OK;
+}
+
+template <typename T>
+int noalloc_launch(const void *Q, const void *K, float *scores, float2 *stats, int units, int M, int N, int d,
+                   size_t k_unit_rows, cudaStream_t stream)
+{
+    const size_t smem = simt_smem_bytes(d);
+    IPOT_CUDA(cudaFuncSetAttribute(cap_row_stats<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)simt_smem_bytes(256)));
+    IPOT_CUDA(cudaFuncSetAttribute(cap_column_sums<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)simt_smem_bytes(256)));
+    const float scale_log2e = (float)(1.4426950408889634 / std::sqrt((double)d));
+    dim3 g1((M + kSimtRows - 1) / kSimtRows, units), g2((N + kSimtKeys - 1) / kSimtKeys, units);
+    cap_row_stats<T><<<g1, kSimtThreads, smem, stream>>>((const T *)Q, (const T *)K, stats, M, N, d, k_unit_rows * d, scale_log2e);
+    cap_column_sums<T><<<g2, kSimtThreads, smem, stream>>>((const T *)Q, (const T *)K, stats, scores, M, N, d, k_unit_rows * d, scale_log2e);
+    IPOT_CUDA(cudaGetLastError());
+    return IPOT_OK;
+}
+}  // namespace
+
+extern "C" int ipot_cap_scores_noalloc(const void *Q, const void *K, float *scores, int units, int rows, int N, int d,
+                                       int k_unit_rows, int dtype, void *cuda_stream)
+{
+    if (!Q || !K || !scores || !aligned16(Q) || !aligned16(K) || (reinterpret_cast<uintptr_t>(scores) & 3u))
+        return IPOT_E_INVALID;
+    if (units < 1 || rows < 1 || N < 1 || k_unit_rows < N || d < 32 || d > 256 || d % 8) return IPOT_E_INVALID;
+    if (dtype != IPOT_BF16 && dtype != IPOT_F32) return IPOT_E_INVALID;
+    if ((long long)units * rows > IPOT_NOALLOC_MAX_ROWS) return IPOT_E_LIMIT;
+    float2 *stats = nullptr;
+    int rc = noalloc_scratch(&stats);
+    if (rc != IPOT_OK) return rc;
+    // every statistics entry that the second launch reads is written by the first one,
+    // so nothing left behind by an earlier call needs clearing
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    return dtype == IPOT_F32
+               ? noalloc_launch<float>(Q, K, scores, stats, units, rows, N, d, (size_t)k_unit_rows, stream)
+               : noalloc_launch<__nv_bfloat16>(Q, K, scores, stats, units, rows, N, d, (size_t)k_unit_rows, stream);
+}

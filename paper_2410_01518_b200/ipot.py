@@ -16,7 +16,8 @@ import os
 
 from . import build as _build
 
-IPOT_OK, IPOT_E_INVALID, IPOT_E_STATE, IPOT_E_NOMEM, IPOT_E_CUDA, IPOT_E_TIMEOUT, IPOT_E_BOUNDS = 0, -1, -2, -3, -4, -5, -6
+IPOT_OK, IPOT_E_INVALID, IPOT_E_STATE, IPOT_E_NOMEM, IPOT_E_CUDA, IPOT_E_TIMEOUT, IPOT_E_BOUNDS, IPOT_E_LIMIT = 0, -1, -2, -3, -4, -5, -6, -7
+IPOT_NOALLOC_MAX_ROWS = 65536
 IPOT_BF16, IPOT_F32 = 0, 1
 IPOT_SCORER_AUTO, IPOT_SCORER_SIMT, IPOT_SCORER_TENSOR = 0, 1, 2
 
@@ -26,7 +27,7 @@ SYMBOLS = [
     "ipot_set_scorer", "ipot_reset", "ipot_append_chunk", "ipot_append_chunk_host",
     "ipot_score_and_compress", "ipot_score_and_compress_host", "ipot_score_only", "ipot_view",
     "ipot_last_indices", "ipot_last_scores", "ipot_sync_status", "ipot_set_profiling",
-    "ipot_kernel_ms", "ipot_launch_count", "ipot_strerror",
+    "ipot_kernel_ms", "ipot_launch_count", "ipot_strerror", "ipot_cap_scores_noalloc",
 ]
 
 
@@ -78,6 +79,7 @@ def lib() -> C.CDLL:
         L.ipot_kernel_ms.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(ip), C.POINTER(ip)]
         L.ipot_launch_count.argtypes = [vp, C.POINTER(C.c_longlong)]
         L.ipot_strerror.argtypes = [ip]
+        L.ipot_cap_scores_noalloc.argtypes = [vp, vp, vp, ip, ip, ip, ip, ip, ip, vp]
         L.ipot_strerror.restype = C.c_char_p
         for s in SYMBOLS:
             if s != "ipot_strerror":
@@ -201,6 +203,14 @@ def ipot_launch_count(h) -> int:
     n = C.c_longlong()
     _check(lib().ipot_launch_count(h, C.byref(n)), "ipot_launch_count")
     return n.value
+
+
+def ipot_cap_scores_noalloc(Q, K, scores, units, rows, N, d, k_unit_rows, dtype, stream=None) -> None:
+    """CaP scores for callers that may not allocate device memory: Q [units][rows][d], K
+    [units][k_unit_rows][d] (first N rows scored) -> scores [units][N] f32, all device buffers of
+    the caller.  Scratch is a fixed array inside the library (units * rows <= IPOT_NOALLOC_MAX_ROWS)."""
+    _check(lib().ipot_cap_scores_noalloc(_ptr(Q), _ptr(K), _ptr(scores), units, rows, N, d, k_unit_rows, dtype,
+                                         stream), "ipot_cap_scores_noalloc")
 
 
 def device_array(addr: int, shape, dtype, device="cuda"):
