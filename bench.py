@@ -172,9 +172,12 @@ def main():
     ap.add_argument("--workload", default="cfg3", choices=sorted(WORKLOADS))
     ap.add_argument("--scorer", default="auto", choices=["auto", "simt", "tensor"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (profiling small cases)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     cfg = inputs.CONFIGS[WORKLOADS[args.workload]]
+    if args.layers > 0:
+        cfg = cfg.with_layers(args.layers)
     if args.impl == "reference":
         run_reference(args, cfg)
         return

@@ -10,7 +10,12 @@ from parity import compare_cycle, from_dev_bits, gpu_cycle, make_pot, read_resul
 
 pytestmark = pytest.mark.gpu
 
-SCORERS = [ipot.IPOT_SCORER_SIMT]
+SCORERS = [ipot.IPOT_SCORER_SIMT, ipot.IPOT_SCORER_TENSOR]
+
+
+def tensor_scorer_applies(cfg, n=None):
+    """The tcgen05 scorer takes bf16, d = 128 and pots of at most 4096 rows."""
+    return cfg.dtype == "bf16" and cfg.d == 128 and (n or cfg.pot_size) <= 4096
 
 
 def test_config1_tiny_f32_all_units():
@@ -21,10 +26,11 @@ def test_config1_tiny_f32_all_units():
     assert n == cfg.units and same == n
 
 
-def test_config2_mistral_layer_bf16_all_units():
+@pytest.mark.parametrize("scorer", SCORERS)
+def test_config2_mistral_layer_bf16_all_units(scorer):
     cfg = inputs.CONFIGS[2]
     t = inputs.make_cycle(cfg)
-    gpu = gpu_cycle(cfg, t, ipot.IPOT_SCORER_SIMT)
+    gpu = gpu_cycle(cfg, t, scorer)
     same, n = compare_cycle(cfg, t, gpu)
     assert n == cfg.units and same >= n - 1  # at most one unit may sit on a tie
 
@@ -47,10 +53,57 @@ SMALL = [
 @pytest.mark.parametrize("scorer", SCORERS)
 def test_small_random_shapes(case, scorer):
     cfg = inputs.small_config(cfg_id=200 + case, **SMALL[case])
+    if scorer == ipot.IPOT_SCORER_TENSOR and not tensor_scorer_applies(cfg):
+        h = make_pot(cfg)
+        try:  # the tensor scorer must refuse, not fall back
+            t = inputs.make_cycle(cfg)
+            ipot.ipot_set_scorer(h, scorer)
+            ipot.ipot_append_chunk(h, to_dev(t["K"], cfg.dtype), to_dev(t["V"], cfg.dtype), cfg.pot_size)
+            rc = ipot.lib().ipot_score_only(h, to_dev(t["Q"], cfg.dtype).data_ptr(), cfg.cap_rows, None)
+            assert rc == ipot.IPOT_E_INVALID
+        finally:
+            ipot.ipot_destroy(h)
+        return
     t = inputs.make_cycle(cfg)
     gpu = gpu_cycle(cfg, t, scorer)
     same, n = compare_cycle(cfg, t, gpu)
     assert n == cfg.units and same >= n - 1
+
+
+TENSOR_SHAPES = [
+    # (pot_size, rows used, cap_rows, Hq, Hkv, layers, batch): cluster sizes 1..8, ragged slabs, 1-3 row blocks
+    (512, 512, 32, 4, 1, 1, 1), (640, 513, 16, 8, 2, 2, 1), (1536, 1500, 33, 8, 2, 1, 2), (2048, 2048, 64, 8, 2, 3, 1),
+    (3000, 2999, 5, 6, 2, 1, 1), (4096, 3585, 64, 12, 2, 2, 1), (4096, 4096, 32, 32, 8, 5, 1), (300, 129, 1, 1, 1, 1, 1),
+]
+
+
+@pytest.mark.parametrize("case", range(len(TENSOR_SHAPES)))
+def test_tensor_scorer_shapes(case):
+    pot, n, P, Hq, Hkv, L, B = TENSOR_SHAPES[case]
+    cfg = inputs.small_config(cfg_id=400 + case, pot_size=pot, keep=n // 2, nuc_slots=n // 4, cap_rows=P, Hq=Hq,
+                              Hkv=Hkv, d=128, dtype="bf16", layers=L, batch=B)
+    t = inputs.make_cycle(cfg)
+    gpu = gpu_cycle(cfg, t, ipot.IPOT_SCORER_TENSOR, n=n)
+    same, cnt = compare_cycle(cfg, t, gpu, n=n)
+    assert cnt == cfg.units and same >= cnt - 1
+    simt = gpu_cycle(cfg, t, ipot.IPOT_SCORER_SIMT, n=n)
+    np.testing.assert_allclose(gpu[0], simt[0], rtol=2e-5, atol=1e-30)  # the two GPU scorers agree far inside 1e-3
+
+
+def test_config3_full_size_sampled_units():
+    """All 32 layers in one call (the launch the benchmark times); the checker follows 12 sampled units."""
+    cfg = inputs.CONFIGS[3]
+    K0, V0 = inputs.make_kv(cfg, 2048, chunk=0)
+    K1, V1 = inputs.make_kv(cfg, 2048, chunk=1)
+    t = {"K": np.concatenate([K0, K1], axis=3), "V": np.concatenate([V0, V1], axis=3),
+         "Q": inputs.make_q(cfg, 1), "aux": inputs.make_aux(cfg, 1)}
+    gpu = gpu_cycle(cfg, t, ipot.IPOT_SCORER_AUTO)
+    units = np.linspace(0, cfg.units - 1, 12).astype(np.int32)
+    same, cnt = compare_cycle(cfg, t, gpu, units=units)
+    assert cnt == 12 and same >= 11
+    u, idx = gpu[0], gpu[1]
+    assert np.abs(u.sum(axis=1) - cfg.G * cfg.cap_rows).max() < 2e-2      # holds at any size
+    assert (np.diff(idx, axis=1) > 0).all() and idx.min() >= 0 and idx.max() < cfg.pot_size
 
 
 def test_partially_filled_pot():
