@@ -14,8 +14,8 @@ SCORERS = [ipot.IPOT_SCORER_SIMT, ipot.IPOT_SCORER_TENSOR]
 
 
 def tensor_scorer_applies(cfg, n=None):
-    """The tcgen05 scorer takes bf16, d = 128 and pots of at most 4096 rows."""
-    return cfg.dtype == "bf16" and cfg.d == 128 and (n or cfg.pot_size) <= 4096
+    """The tcgen05 scorer takes bf16 with d = 128 (any pot size the library accepts)."""
+    return cfg.dtype == "bf16" and cfg.d == 128
 
 
 def test_config1_tiny_f32_all_units():
@@ -71,9 +71,11 @@ def test_small_random_shapes(case, scorer):
 
 
 TENSOR_SHAPES = [
-    # (pot_size, rows used, cap_rows, Hq, Hkv, layers, batch): cluster sizes 1..8, ragged slabs, 1-3 row blocks
+    # (pot_size, rows used, cap_rows, Hq, Hkv, layers, batch): 1..64 slabs per item, ragged slabs, 1-4 row blocks,
+    # fewer and more tasks than SMs
     (512, 512, 32, 4, 1, 1, 1), (640, 513, 16, 8, 2, 2, 1), (1536, 1500, 33, 8, 2, 1, 2), (2048, 2048, 64, 8, 2, 3, 1),
     (3000, 2999, 5, 6, 2, 1, 1), (4096, 3585, 64, 12, 2, 2, 1), (4096, 4096, 32, 32, 8, 5, 1), (300, 129, 1, 1, 1, 1, 1),
+    (8192, 8192, 64, 8, 2, 1, 2), (16384, 16001, 64, 8, 1, 1, 2), (5000, 4097, 40, 4, 1, 20, 1),
 ]
 
 
