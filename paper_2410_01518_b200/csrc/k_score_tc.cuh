@@ -11,20 +11,22 @@
 //            shared memory in the 128-byte-swizzled K-major layout (2 stages);
 //   tcgen05  S = Q K^T (128 x 256 fp32) accumulates in one of two 256-column tensor
 //            memory buffers: the logits never leave the SM;
-//   pass 1   (warps 2-5, one thread per query row) slab maximum, e = 2^(x - max)
-//            written back over the logits, slab sum; (max, sum) of every row goes to
-//            a small global array and the item's arrival counter is bumped;
-//   pass 2   (warps 6-9) once all slabs of the item have arrived - normally long
-//            before, since the CTA has meanwhile run pass 1 of its next task - the
-//            row's global maximum m and denominator l are combined from the slabs'
-//            statistics and u_j = sum_i e_ij 2^(max_slab,i - m_i) / l_i is formed
-//            as a weighted column sum (per-warp shared-memory transpose, then across
-//            the four row quarters) and stored: 256 floats per task.
+//   pass 1   (warps 2-9, two threads per query row, 128 columns each) maximum,
+//            e = 2^(x - max) written back over the logits, sum; the row's slab
+//            statistics (max, sum) go to a small global array, one 8-byte store per
+//            row whose sum carries the launch's sign as a "fresh" mark;
+//   pass 2   (warps 10-17) each thread reads its row's statistics of all slabs of
+//            the item, re-reading until every one is fresh - normally they are, as
+//            the CTA has meanwhile run pass 1 of its next task - and combines them
+//            into the row's global maximum m and denominator l; then
+//            u_j = sum_i e_ij 2^(max_i - m_i) / l_i is formed as a weighted column
+//            sum (per-warp shared-memory transpose, then across the four row
+//            quarters) and stored: 256 floats per task.
 //
 // Blocks of one grid wait on each other (pass 2 needs the other slabs' statistics),
 // so the grid is launched cooperatively with at most one CTA per SM: all of it is
 // resident.  A CTA publishes pass 1 of task t+1 before it waits for task t, so the
-// waits cannot form a cycle.  Every wait (mbarrier or counter) is bounded; one that
+// waits cannot form a cycle.  Every wait (mbarrier or statistics) is bounded; one that
 // runs out records IPOT_E_TIMEOUT in the status word and lets the CTA run to its
 // normal end with tensor memory released.
 #pragma once
@@ -37,7 +39,7 @@
 
 namespace ipotk {
 
-constexpr int kTcThreads = 320;      // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-5: pass 1, warps 6-9: pass 2
+constexpr int kTcThreads = 576;      // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-9: pass 1, warps 10-17: pass 2
 constexpr int kTcRows = 128;         // query rows per item (TMEM lanes)
 constexpr int kTcSlab = 256;         // keys per task (TMEM columns per buffer)
 constexpr int kTcD = 128;
@@ -48,11 +50,11 @@ constexpr uint32_t kTcSpinLimit = 1u << 22;                  // try_wait / poll 
 
 // shared-memory carve-up (bytes from the 1024-aligned base)
 constexpr uint32_t kTcOffStage = 0;                                        // [2] { Q, K }
-constexpr uint32_t kTcOffTbuf = 2 * kTcStageBytes;                         // [4 warps][32][36] float
-constexpr uint32_t kTcOffColpart = kTcOffTbuf + 4 * 32 * 36 * 4;           // [4][256] float
-constexpr uint32_t kTcOffLocm = kTcOffColpart + 4 * kTcSlab * 4;           // [2][128] float
-constexpr uint32_t kTcOffFrow = kTcOffLocm + 2 * kTcRows * 4;              // [4 warps][32] float
-constexpr uint32_t kTcOffBar = kTcOffFrow + 4 * 32 * 4;
+constexpr uint32_t kTcOffTbuf = 2 * kTcStageBytes;                         // [8 warps][16][36] float
+constexpr uint32_t kTcOffColpart = kTcOffTbuf + 8 * 16 * 36 * 4;           // [4][256] float
+constexpr uint32_t kTcOffHalf = kTcOffColpart + 4 * kTcSlab * 4;           // [2 buffers][2 halves][128] float2
+constexpr uint32_t kTcOffFrow = kTcOffHalf + 2 * 2 * kTcRows * 8;          // [8 warps][32] float
+constexpr uint32_t kTcOffBar = kTcOffFrow + 8 * 32 * 4;
 constexpr uint32_t kTcSmemBytes = kTcOffBar + 128 + 1024;                  // + alignment slack
 
 enum { kBarFull = 0, kBarEmpty = 2, kBarSFull = 4, kBarEReady = 6, kBarTEmpty = 8, kBarCount = 10 };
@@ -60,8 +62,8 @@ enum { kBarFull = 0, kBarEmpty = 2, kBarSFull = 4, kBarEReady = 6, kBarTEmpty = 
 struct TcParams {
     float *scores;        // partial array p (query rows 128p ...) at scores + p * part_stride, unit stride N
     size_t part_stride;
-    float2 *stats;        // [items][slabs][128] (max in log2 units, sum)
-    unsigned int *arrived;  // [items], zero at launch
+    float2 *stats;        // [items][slabs][128] (max in log2 units, sum * sign); all of the other sign or 0 at launch
+    float sign;           // +1 or -1: this launch's "fresh" mark
     int *status;
     int N, M, mtiles, slabs, tasks;
     float scale_log2e;
@@ -139,6 +141,23 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32])
           "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
         : "r"(taddr) : "memory");
 }
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld16(uint32_t (&v)[16])
+{
+    asm volatile(
+        "tcgen05.wait::ld.sync.aligned;"
+        : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]),
+          "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]), "+r"(v[15])
+        :: "memory");
+}
 // Waits for this thread's outstanding TMEM loads.  The loaded registers are passed
 // through so that no use of them can be scheduled ahead of the wait.
 __device__ __forceinline__ void tmem_wait_ld(uint32_t (&v)[32])
@@ -166,9 +185,21 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 template <int kId>
-__device__ __forceinline__ void group_bar_sync()  // 128-thread named barrier of one epilogue group
+__device__ __forceinline__ void group_bar_sync()  // 256-thread named barrier of one epilogue group
 {
-    asm volatile("bar.sync %0, 128;" ::"n"(kId) : "memory");
+    asm volatile("bar.sync %0, 256;" ::"n"(kId) : "memory");
+}
+// The slab statistics are exchanged between CTAs with single 8-byte relaxed accesses at gpu scope:
+// one store publishes (max, marked sum) together, and a reader sees either the old or the new pair.
+__device__ __forceinline__ float2 ld_gpu_f32x2(const float2 *p)
+{
+    float2 v;
+    asm volatile("ld.relaxed.gpu.global.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_gpu_f32x2(float2 *p, float a, float b)
+{
+    asm volatile("st.relaxed.gpu.global.v2.f32 [%0], {%1, %2};" ::"l"(p), "f"(a), "f"(b) : "memory");
 }
 __device__ __forceinline__ float ex2(float x)
 {
@@ -176,11 +207,109 @@ __device__ __forceinline__ float ex2(float x)
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-__device__ __forceinline__ unsigned int ld_acquire_gpu(const unsigned int *p)
+__device__ __forceinline__ float max3(float a, float b, float c)
 {
-    unsigned int v;
-    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-    return v;
+    float y;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
+    return y;
+}
+
+// Maximum of 32 logits folded into four independent running maxima (no long dependency chain).
+template <bool kFull>
+__device__ __forceinline__ void chunk_max(const uint32_t (&v)[32], int col0, int nvalid, float (&mx)[4])
+{
+    if (kFull) {
+#pragma unroll
+        for (int i = 0; i < 32; i += 8) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) mx[j] = max3(mx[j], __uint_as_float(v[i + 2 * j]), __uint_as_float(v[i + 2 * j + 1]));
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+            if (col0 + i < nvalid) mx[i & 3] = fmaxf(mx[i & 3], __uint_as_float(v[i]));
+    }
+}
+
+// v <- 2^(v c - mxc) (0 beyond nvalid); the new values are also added into four packed running sums.
+template <bool kFull>
+__device__ __forceinline__ void chunk_exp(uint32_t (&v)[32], int col0, int nvalid, float c, float mxc, float2 (&sum)[4])
+{
+    const float2 c2 = make_float2(c, c), nm2 = make_float2(-mxc, -mxc);
+#pragma unroll
+    for (int i = 0; i < 32; i += 2) {
+        const float2 x = __ffma2_rn(make_float2(__uint_as_float(v[i]), __uint_as_float(v[i + 1])), c2, nm2);
+        float2 e2 = make_float2(ex2(x.x), ex2(x.y));
+        if (!kFull) {
+            if (col0 + i >= nvalid) e2.x = 0.f;
+            if (col0 + i + 1 >= nvalid) e2.y = 0.f;
+        }
+        sum[(i >> 1) & 3] = __fadd2_rn(sum[(i >> 1) & 3], e2);
+        v[i] = __float_as_uint(e2.x);
+        v[i + 1] = __float_as_uint(e2.y);
+    }
+}
+
+// Pass 1 for one query row over 128 columns starting at col0: returns their maximum (log2 units) and
+// sum of e = 2^(x - max), and leaves e in tensor memory.  TMEM loads run one 32-column chunk ahead of
+// the arithmetic.  With no valid column the maximum is -inf, the sum 0 and zeros are stored.
+template <bool kFull>
+__device__ __forceinline__ void pass1_row(uint32_t trow, int col0, int nvalid, float c, float &mxc_out, float &sum_out)
+{
+    uint32_t va[32], vb[32];
+    float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+    tmem_ld32(trow, va);
+#pragma unroll 1
+    for (int ch = 0; ch < 4; ch += 2) {
+        tmem_wait_ld(va);
+        tmem_ld32(trow + (ch + 1) * 32, vb);
+        chunk_max<kFull>(va, col0 + ch * 32, nvalid, mx);
+        tmem_wait_ld(vb);
+        if (ch + 2 < 4) tmem_ld32(trow + (ch + 2) * 32, va);
+        chunk_max<kFull>(vb, col0 + (ch + 1) * 32, nvalid, mx);
+    }
+    const float mxr = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+    const float mxc = (mxr == -INFINITY) ? 0.f : mxr * c;
+    float2 sum[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+    tmem_ld32(trow, va);
+#pragma unroll 1
+    for (int ch = 0; ch < 4; ch += 2) {
+        tmem_wait_ld(va);
+        tmem_ld32(trow + (ch + 1) * 32, vb);
+        chunk_exp<kFull>(va, col0 + ch * 32, nvalid, c, mxc, sum);
+        tmem_st32(trow + ch * 32, va);
+        tmem_wait_ld(vb);
+        if (ch + 2 < 4) tmem_ld32(trow + (ch + 2) * 32, va);
+        chunk_exp<kFull>(vb, col0 + (ch + 1) * 32, nvalid, c, mxc, sum);
+        tmem_st32(trow + (ch + 1) * 32, vb);
+    }
+    tmem_wait_st();
+    const float2 s01 = __fadd2_rn(sum[0], sum[1]), s23 = __fadd2_rn(sum[2], sum[3]);
+    mxc_out = (mxr == -INFINITY) ? -INFINITY : mxc;
+    sum_out = (s01.x + s01.y) + (s23.x + s23.y);
+}
+
+// One 16-column chunk of pass 2 for one warp (32 rows): the chunk is transposed through the warp's
+// shared-memory tile ([column][row], row stride 36 floats); lane j < 16 then forms
+// sum_{r<16} fr[r] e[r][j], lane j >= 16 the same over rows 16..31 of column j - 16, and the two halves
+// are added.  fr2 holds this lane's 16 row weights as 8 pairs.  Returns the column sum in lanes 0..15.
+__device__ __forceinline__ float pass2_chunk(const uint32_t (&v)[16], float *tbuf, int lane, const float2 (&fr2)[8])
+{
+#pragma unroll
+    for (int cidx = 0; cidx < 16; ++cidx) tbuf[cidx * 36 + lane] = __uint_as_float(v[cidx]);
+    __syncwarp();
+    const float *src = tbuf + (lane & 15) * 36 + (lane & 16);
+    float2 acc[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+#pragma unroll
+    for (int k4 = 0; k4 < 4; ++k4) {
+        const float4 t = *reinterpret_cast<const float4 *>(src + 4 * k4);
+        acc[0] = __ffma2_rn(fr2[2 * k4], make_float2(t.x, t.y), acc[0]);
+        acc[1] = __ffma2_rn(fr2[2 * k4 + 1], make_float2(t.z, t.w), acc[1]);
+    }
+    __syncwarp();
+    const float2 a = __fadd2_rn(acc[0], acc[1]);
+    const float part = a.x + a.y;
+    return part + __shfl_xor_sync(0xffffffffu, part, 16);
 }
 
 // Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128
@@ -213,8 +342,8 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
             mbar_init(bar(kBarFull + b), 1);
             mbar_init(bar(kBarEmpty + b), 1);
             mbar_init(bar(kBarSFull + b), 1);
-            mbar_init(bar(kBarEReady + b), 128);
-            mbar_init(bar(kBarTEmpty + b), 128);
+            mbar_init(bar(kBarEReady + b), 256);
+            mbar_init(bar(kBarTEmpty + b), 256);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -268,160 +397,113 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
             }
         }
         __syncwarp();
-    } else if (warp < 6) {
-        // ---------------------------------------------------------------- pass 1 (128 threads, one per query row)
+    } else if (warp < 10) {
+        // ---------------------------------------------------------------- pass 1 (256 threads: row x column half)
         const int q = warp & 3;                 // TMEM lane quarter this warp may touch
+        const int half = (warp - 2) >> 2;       // which 128 columns of the slab
         const int row = q * 32 + lane;
-        const int gt = threadIdx.x - 64;        // 0..127 within the group
-        float *locm = reinterpret_cast<float *>(gbase + kTcOffLocm);
+        float2 *halfst = reinterpret_cast<float2 *>(gbase + kTcOffHalf);
         const float c = prm.scale_log2e;
         uint32_t k = 0;
         for (int task = blockIdx.x; task < prm.tasks; task += gridDim.x, ++k) {
             const int item = task / tasks_per_item, slab = task - item * tasks_per_item;
             const int nvalid = min(kTcSlab, prm.N - slab * kTcSlab);
             const uint32_t b = k & 1, ph = (k >> 1) & 1;
-            const uint32_t trow = tmem + ((uint32_t)(q * 32) << 16) + b * kTcSlab;
+            const uint32_t trow = tmem + ((uint32_t)(q * 32) << 16) + b * kTcSlab + half * 128;
             mbar_wait(bar(kBarSFull + b), ph, ab, prm.status);
             tc_fence_after();
-
-            // ---- maximum over the valid columns (loads run one chunk ahead of the compares)
-            float mx = -INFINITY;
-            {
-                uint32_t va[32], vb[32];
-                tmem_ld32(trow, va);
-#pragma unroll 1
-                for (int ch = 0; ch < 8; ch += 2) {
-                    tmem_wait_ld(va);
-                    tmem_ld32(trow + (ch + 1) * 32, vb);
-#pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        if (ch * 32 + i < nvalid) mx = fmaxf(mx, __uint_as_float(va[i]));
-                    tmem_wait_ld(vb);
-                    if (ch + 2 < 8) tmem_ld32(trow + (ch + 2) * 32, va);
-#pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        if ((ch + 1) * 32 + i < nvalid) mx = fmaxf(mx, __uint_as_float(vb[i]));
-                }
-            }
-            // ---- e = 2^((s - max) c) over the logits, in place; row sum
-            const float mxc = mx * c;  // finite: every slab has at least one valid key
-            float sum = 0.f;
-            {
-                uint32_t va[32], vb[32];
-                tmem_ld32(trow, va);
-#pragma unroll 1
-                for (int ch = 0; ch < 8; ch += 2) {
-                    tmem_wait_ld(va);
-                    tmem_ld32(trow + (ch + 1) * 32, vb);
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        const float ev = (ch * 32 + i < nvalid) ? ex2(fmaf(__uint_as_float(va[i]), c, -mxc)) : 0.f;
-                        sum += ev;
-                        va[i] = __float_as_uint(ev);
-                    }
-                    tmem_st32(trow + ch * 32, va);
-                    tmem_wait_ld(vb);
-                    if (ch + 2 < 8) tmem_ld32(trow + (ch + 2) * 32, va);
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        const float ev = ((ch + 1) * 32 + i < nvalid) ? ex2(fmaf(__uint_as_float(vb[i]), c, -mxc)) : 0.f;
-                        sum += ev;
-                        vb[i] = __float_as_uint(ev);
-                    }
-                    tmem_st32(trow + (ch + 1) * 32, vb);
-                }
-            }
-            tmem_wait_st();
-            // ---- publish: the reference of the stored e values for pass 2, the slab statistics for everyone
-            locm[b * kTcRows + row] = mxc;
-            prm.stats[((size_t)item * tasks_per_item + slab) * kTcRows + row] = make_float2(mxc, sum);
+            float mxc, sum;
+            if (nvalid == kTcSlab) pass1_row<true>(trow, half * 128, nvalid, c, mxc, sum);
+            else pass1_row<false>(trow, half * 128, nvalid, c, mxc, sum);
+            // the reference of the stored e values (pass 2 needs it) and this half's sum
+            halfst[(b * 2 + half) * kTcRows + row] = make_float2(mxc, sum);
             tc_fence_before();
             mbar_arrive(bar(kBarEReady + b));
-            group_bar_sync<1>();              // all 128 statistics of the slab are written
-            if (gt == 0) {
-                __threadfence();
-                atomicAdd(&prm.arrived[item], 1u);
+            group_bar_sync<1>();
+            if (half == 0) {  // merge the two halves, publish the slab's statistics of this row
+                const float2 h0 = halfst[(b * 2) * kTcRows + row], h1 = halfst[(b * 2 + 1) * kTcRows + row];
+                const float m = fmaxf(h0.x, h1.x);  // half 0 always holds a valid key
+                const float l = h0.y * ex2(h0.x - m) + (h1.x == -INFINITY ? 0.f : h1.y * ex2(h1.x - m));
+                st_gpu_f32x2(&prm.stats[((size_t)item * tasks_per_item + slab) * kTcRows + row], m, l * prm.sign);
             }
         }
     } else {
-        // ---------------------------------------------------------------- pass 2 (128 threads)
+        // ---------------------------------------------------------------- pass 2 (256 threads)
         const int q = warp & 3;
-        const int w = warp - 6;                 // 0..3
+        const int w = warp - 10;                // 0..7
+        const int half = w >> 2;
         const int row = q * 32 + lane;
-        const int gt = threadIdx.x - 192;       // 0..127 within the group
-        float *tbuf = reinterpret_cast<float *>(gbase + kTcOffTbuf) + w * (32 * 36);
+        const int gt = threadIdx.x - 320;       // 0..255 within the group
+        float *tbuf = reinterpret_cast<float *>(gbase + kTcOffTbuf) + w * (16 * 36);
         float *colpart = reinterpret_cast<float *>(gbase + kTcOffColpart);
-        const float *locm = reinterpret_cast<const float *>(gbase + kTcOffLocm);
+        const float2 *halfst = reinterpret_cast<const float2 *>(gbase + kTcOffHalf);
         float *frow = reinterpret_cast<float *>(gbase + kTcOffFrow) + w * 32;
+        const float sgn = prm.sign;
         uint32_t k = 0;
         for (int task = blockIdx.x; task < prm.tasks; task += gridDim.x, ++k) {
             const int item = task / tasks_per_item, slab = task - item * tasks_per_item;
             const int unit = item / prm.mtiles, mt = item - unit * prm.mtiles;
             const int nvalid = min(kTcSlab, prm.N - slab * kTcSlab);
             const uint32_t b = k & 1, ph = (k >> 1) & 1;
-            const uint32_t trow = tmem + ((uint32_t)(q * 32) << 16) + b * kTcSlab;
+            const uint32_t trow = tmem + ((uint32_t)(q * 32) << 16) + b * kTcSlab + half * 128;
             mbar_wait(bar(kBarEReady + b), ph, ab, prm.status);
             tc_fence_after();
 
-            // ---- wait until every slab of the item has published its statistics
-            if (gt == 0) {
-                bool ok = false;
-                for (uint32_t i = 0; i < kTcSpinLimit; ++i) {
-                    if (ld_acquire_gpu(&prm.arrived[item]) >= (unsigned int)tasks_per_item) { ok = true; break; }
-                    if (*ab) break;
-                    __nanosleep(32);
-                }
-                if (!ok && !*ab) {
-                    *ab = 1;
-                    set_status(prm.status, kStatusTimeout);
-                }
-                __threadfence();
-            }
-            group_bar_sync<2>();
+            // ---- this row's statistics of every slab of the item; re-read until all carry this launch's mark
             const float2 *st = prm.stats + (size_t)item * tasks_per_item * kTcRows + row;
-            float m = -INFINITY;
-            for (int s = 0; s < tasks_per_item; ++s) m = fmaxf(m, __ldcg(&st[(size_t)s * kTcRows]).x);
-            float l = 0.f;
-            for (int s = 0; s < tasks_per_item; ++s) {
-                const float2 s2 = __ldcg(&st[(size_t)s * kTcRows]);
-                l += s2.y * ex2(s2.x - m);
+            float m = -INFINITY, l = 0.f;
+            for (int s0 = 0; s0 < tasks_per_item; s0 += 16) {
+                float2 sv[16];
+                uint32_t tries = 0;
+                bool fresh;
+                do {
+                    fresh = true;
+#pragma unroll
+                    for (int s = 0; s < 16; ++s) {
+                        sv[s] = (s0 + s < tasks_per_item) ? ld_gpu_f32x2(&st[(size_t)(s0 + s) * kTcRows]) : make_float2(-INFINITY, sgn);
+                        fresh = fresh && (sv[s].y * sgn > 0.f);
+                    }
+                    if (!fresh && ((++tries > kTcSpinLimit / 64) || *ab)) {
+                        if (!*ab) {
+                            *ab = 1;
+                            set_status(prm.status, kStatusTimeout);
+                        }
+                        break;
+                    }
+                    if (!fresh) __nanosleep(100);
+                } while (!fresh);
+                float mb = m;
+#pragma unroll
+                for (int s = 0; s < 16; ++s) mb = fmaxf(mb, sv[s].x);
+                l = (m == -INFINITY) ? 0.f : l * ex2(m - mb);
+#pragma unroll
+                for (int s = 0; s < 16; ++s) l = fmaf(fabsf(sv[s].y), ex2(sv[s].x - mb), l);
+                m = mb;
             }
             const bool row_valid = mt * kTcRows + row < prm.M;
-            const float f = row_valid ? ex2(locm[b * kTcRows + row] - m) / l : 0.f;
+            const float mine = halfst[(b * 2 + half) * kTcRows + row].x;
+            const float f = (row_valid && mine != -INFINITY) ? ex2(mine - m) / l : 0.f;
             frow[lane] = f;
             __syncwarp();
-            float fr[32];
+            float2 fr2[8];  // the weights of the 16 rows this lane sums over
 #pragma unroll
-            for (int i = 0; i < 32; ++i) fr[i] = frow[i];
+            for (int i = 0; i < 8; ++i) fr2[i] = *reinterpret_cast<const float2 *>(frow + (lane & 16) + 2 * i);
+            __syncwarp();
 
-            // ---- weighted column sums over this warp's 32 rows
+            // ---- weighted column sums over this warp's 32 rows, 16 columns at a time
             {
-                uint32_t va[32], vb[32];
-                tmem_ld32(trow, va);
+                uint32_t va[16], vb[16];
+                tmem_ld16(trow, va);
 #pragma unroll 1
                 for (int ch = 0; ch < 8; ch += 2) {
-                    tmem_wait_ld(va);
-                    tmem_ld32(trow + (ch + 1) * 32, vb);
-#pragma unroll
-                    for (int i = 0; i < 32; i += 4)
-                        *reinterpret_cast<uint4 *>(tbuf + lane * 36 + i) = make_uint4(va[i], va[i + 1], va[i + 2], va[i + 3]);
-                    __syncwarp();
-                    float acc = 0.f;
-#pragma unroll
-                    for (int r = 0; r < 32; ++r) acc = fmaf(fr[r], tbuf[r * 36 + lane], acc);
-                    __syncwarp();
-                    colpart[q * kTcSlab + ch * 32 + lane] = acc;
-                    tmem_wait_ld(vb);
-                    if (ch + 2 < 8) tmem_ld32(trow + (ch + 2) * 32, va);
-#pragma unroll
-                    for (int i = 0; i < 32; i += 4)
-                        *reinterpret_cast<uint4 *>(tbuf + lane * 36 + i) = make_uint4(vb[i], vb[i + 1], vb[i + 2], vb[i + 3]);
-                    __syncwarp();
-                    acc = 0.f;
-#pragma unroll
-                    for (int r = 0; r < 32; ++r) acc = fmaf(fr[r], tbuf[r * 36 + lane], acc);
-                    __syncwarp();
-                    colpart[q * kTcSlab + (ch + 1) * 32 + lane] = acc;
+                    tmem_wait_ld16(va);
+                    tmem_ld16(trow + (ch + 1) * 16, vb);
+                    float u = pass2_chunk(va, tbuf, lane, fr2);
+                    if (lane < 16) colpart[q * kTcSlab + half * 128 + ch * 16 + lane] = u;
+                    tmem_wait_ld16(vb);
+                    if (ch + 2 < 8) tmem_ld16(trow + (ch + 2) * 16, va);
+                    u = pass2_chunk(vb, tbuf, lane, fr2);
+                    if (lane < 16) colpart[q * kTcSlab + half * 128 + (ch + 1) * 16 + lane] = u;
                 }
             }
             tc_fence_before();
@@ -429,9 +511,11 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
 
             // ---- add the four row quarters, store this task's scores
             group_bar_sync<2>();
-            float *out = prm.scores + (size_t)mt * prm.part_stride + (size_t)unit * prm.N + slab * kTcSlab;
-            for (int col = gt; col < nvalid; col += 128)
-                out[col] = (colpart[col] + colpart[kTcSlab + col]) + (colpart[2 * kTcSlab + col] + colpart[3 * kTcSlab + col]);
+            if (gt < nvalid) {
+                float *out = prm.scores + (size_t)mt * prm.part_stride + (size_t)unit * prm.N + slab * kTcSlab;
+                out[gt] = (colpart[gt] + colpart[kTcSlab + gt]) + (colpart[2 * kTcSlab + gt] + colpart[3 * kTcSlab + gt]);
+            }
+            group_bar_sync<2>();                // colpart is rewritten by the next task
         }
     }
 
@@ -455,15 +539,16 @@ struct TcPlan {
     int sm_count = 0;
     int max_items = 0, max_slabs = 0;
     float2 *stats = nullptr;          // [max_items][max_slabs][128]
-    unsigned int *arrived = nullptr;  // [max_items]
+    // "fresh" marking of the statistics: every launch writes all entries of its (items x slabs) layout
+    // with the sign opposite to the previous launch's; a layout change clears the array first
+    float sign = 1.f;
+    int last_items = 0, last_slabs = 0;
 };
 
 inline void tc_plan_destroy(TcPlan &plan)
 {
     cudaFree(plan.stats);
-    cudaFree(plan.arrived);
     plan.stats = nullptr;
-    plan.arrived = nullptr;
     plan.usable = false;
 }
 
@@ -493,8 +578,7 @@ inline void tc_plan_init(TcPlan &plan, const ipot_config_t &cfg, const void *, i
     const int units = cfg.layers * cfg.batch * cfg.Hkv;
     plan.max_items = units * ((G * cfg.max_cap_rows + kTcRows - 1) / kTcRows);
     plan.max_slabs = (cfg.pot_size + kTcSlab - 1) / kTcSlab;
-    if (cudaMalloc(&plan.stats, (size_t)plan.max_items * plan.max_slabs * kTcRows * sizeof(float2)) != cudaSuccess ||
-        cudaMalloc(&plan.arrived, (size_t)plan.max_items * sizeof(unsigned int)) != cudaSuccess) {
+    if (cudaMalloc(&plan.stats, (size_t)plan.max_items * plan.max_slabs * kTcRows * sizeof(float2)) != cudaSuccess) {
         cudaGetLastError();
         tc_plan_destroy(plan);
         return;
@@ -532,15 +616,21 @@ inline int tc_launch(TcPlan &plan, const ipot_config_t &cfg, const void *Q, cons
     if (tc_encode_rows(plan, &mapQ, Q, M, units, (size_t)M, kTcRows) != IPOT_OK) return IPOT_E_CUDA;
     if (tc_encode_rows(plan, &mapK, K, N, units, (size_t)cfg.pot_size, kTcSlab) != IPOT_OK) return IPOT_E_CUDA;
     TcParams prm;
-    prm.scores = scores; prm.part_stride = part_stride; prm.stats = plan.stats; prm.arrived = plan.arrived; prm.status = status;
+    prm.scores = scores; prm.part_stride = part_stride; prm.stats = plan.stats; prm.status = status;
     prm.N = N; prm.M = M; prm.mtiles = mtiles; prm.slabs = (N + kTcSlab - 1) / kTcSlab;
     const int items = units * mtiles;
     prm.tasks = items * prm.slabs;
     prm.scale_log2e = (float)(1.4426950408889634 / sqrt((double)cfg.d));
-    if (cudaMemsetAsync(plan.arrived, 0, (size_t)items * sizeof(unsigned int), stream) != cudaSuccess) {
-        cudaGetLastError();
-        return IPOT_E_CUDA;
+    if (items != plan.last_items || prm.slabs != plan.last_slabs) {
+        if (cudaMemsetAsync(plan.stats, 0, (size_t)items * prm.slabs * kTcRows * sizeof(float2), stream) != cudaSuccess) {
+            cudaGetLastError();
+            return IPOT_E_CUDA;
+        }
+        plan.last_items = items;
+        plan.last_slabs = prm.slabs;
     }
+    plan.sign = -plan.sign;
+    prm.sign = plan.sign;
     cudaLaunchConfig_t lc = {};
     lc.gridDim = dim3(prm.tasks < plan.sm_count ? prm.tasks : plan.sm_count, 1, 1);
     lc.blockDim = dim3(kTcThreads, 1, 1);
