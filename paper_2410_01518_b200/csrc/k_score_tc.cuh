@@ -15,13 +15,16 @@
 //            e = 2^(x - max) written back over the logits, sum; the row's slab
 //            statistics (max, sum) go to a small global array, one 8-byte store per
 //            row whose sum carries the launch's sign as a "fresh" mark;
-//   pass 2   (warps 10-17) each thread reads its row's statistics of all slabs of
-//            the item, re-reading until every one is fresh - normally they are, as
-//            the CTA has meanwhile run pass 1 of its next task - and combines them
-//            into the row's global maximum m and denominator l; then
-//            u_j = sum_i e_ij 2^(max_i - m_i) / l_i is formed as a weighted column
-//            sum (per-warp shared-memory transpose, then across the four row
-//            quarters) and stored: 256 floats per task.
+//   combine  (warps 18-21, one thread per query row) reads the row's statistics of
+//            all slabs of the item, re-reading until every one is fresh - normally
+//            they are, as the CTA has meanwhile started pass 1 of its next task -
+//            and turns them into the row's global maximum m, denominator l and the
+//            weights 2^(max - m) / l of the stored e values;
+//   pass 2   (warps 10-17) u_j = sum_i e_ij 2^(max_i - m_i) / l_i as a weighted
+//            column sum (per-warp shared-memory transpose, then across the four row
+//            quarters), stored: 256 floats per task.
+// The two 128-column halves of a buffer are handed over separately (MMA -> pass 1,
+// pass 2 -> MMA), so the tensor core refills one half while the other is still read.
 //
 // Blocks of one grid wait on each other (pass 2 needs the other slabs' statistics),
 // so the grid is launched cooperatively with at most one CTA per SM: all of it is
@@ -39,25 +42,27 @@
 
 namespace ipotk {
 
-constexpr int kTcThreads = 576;      // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-9: pass 1, warps 10-17: pass 2
+constexpr int kTcThreads = 704;      // warp 0: TMA, 1: MMA + TMEM owner, 2-9: pass 1, 10-17: pass 2, 18-21: combine
 constexpr int kTcRows = 128;         // query rows per item (TMEM lanes)
 constexpr int kTcSlab = 256;         // keys per task (TMEM columns per buffer)
 constexpr int kTcD = 128;
 constexpr uint32_t kTcQBytes = kTcRows * kTcD * 2;           // 32 KiB
 constexpr uint32_t kTcKBytes = kTcSlab * kTcD * 2;           // 64 KiB
 constexpr uint32_t kTcStageBytes = kTcQBytes + kTcKBytes;    // 96 KiB
-constexpr uint32_t kTcSpinLimit = 1u << 22;                  // try_wait / poll rounds before giving up
+constexpr uint32_t kTcSpinLimit = 1u << 18;                  // try_wait / poll rounds before giving up
 
 // shared-memory carve-up (bytes from the 1024-aligned base)
 constexpr uint32_t kTcOffStage = 0;                                        // [2] { Q, K }
-constexpr uint32_t kTcOffTbuf = 2 * kTcStageBytes;                         // [8 warps][16][36] float
-constexpr uint32_t kTcOffColpart = kTcOffTbuf + 8 * 16 * 36 * 4;           // [4][256] float
+constexpr uint32_t kTcTbufStride = 34;                                     // float2 per column pair (32 rows + pad)
+constexpr uint32_t kTcOffTbuf = 2 * kTcStageBytes;                         // [8 warps][8 pairs][34] float2
+constexpr uint32_t kTcOffColpart = kTcOffTbuf + 8 * 8 * kTcTbufStride * 8; // [4][256] float
 constexpr uint32_t kTcOffHalf = kTcOffColpart + 4 * kTcSlab * 4;           // [2 buffers][2 halves][128] float2
-constexpr uint32_t kTcOffFrow = kTcOffHalf + 2 * 2 * kTcRows * 8;          // [8 warps][32] float
-constexpr uint32_t kTcOffBar = kTcOffFrow + 8 * 32 * 4;
-constexpr uint32_t kTcSmemBytes = kTcOffBar + 128 + 1024;                  // + alignment slack
+constexpr uint32_t kTcOffFbuf = kTcOffHalf + 2 * 2 * kTcRows * 8;          // [2 buffers][2 halves][128] float
+constexpr uint32_t kTcOffBar = kTcOffFbuf + 2 * 2 * kTcRows * 4;
+constexpr uint32_t kTcSmemBytes = kTcOffBar + 256 + 1024;                  // + alignment slack
 
-enum { kBarFull = 0, kBarEmpty = 2, kBarSFull = 4, kBarEReady = 6, kBarTEmpty = 8, kBarCount = 10 };
+// barriers: per stage Full, Empty, FReady; per (buffer, half) SFull, EReady, TEmpty at index 2 * buffer + half
+enum { kBarFull = 0, kBarEmpty = 2, kBarFReady = 4, kBarSFull = 6, kBarEReady = 10, kBarTEmpty = 14, kBarCount = 18 };
 
 struct TcParams {
     float *scores;        // partial array p (query rows 128p ...) at scores + p * part_stride, unit stride N
@@ -89,9 +94,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(20000u) : "memory");  // may sleep up to ~20 us per try
     return ok != 0;
 }
 // Bounded wait.  Once any wait of the CTA has run out, later waits return at once.
@@ -289,27 +294,30 @@ __device__ __forceinline__ void pass1_row(uint32_t trow, int col0, int nvalid, f
     sum_out = (s01.x + s01.y) + (s23.x + s23.y);
 }
 
-// One 16-column chunk of pass 2 for one warp (32 rows): the chunk is transposed through the warp's
-// shared-memory tile ([column][row], row stride 36 floats); lane j < 16 then forms
-// sum_{r<16} fr[r] e[r][j], lane j >= 16 the same over rows 16..31 of column j - 16, and the two halves
-// are added.  fr2 holds this lane's 16 row weights as 8 pairs.  Returns the column sum in lanes 0..15.
-__device__ __forceinline__ float pass2_chunk(const uint32_t (&v)[16], float *tbuf, int lane, const float2 (&fr2)[8])
+// One 16-column chunk of pass 2 for one warp (32 rows).  The chunk is transposed through the warp's
+// shared-memory tile as 8 column pairs: tile[pair][row] (float2, row stride 34).  Lane (g, p) = (lane / 8,
+// lane % 8) then forms sum_{r in 8g..8g+7} f_r (e[r][2p], e[r][2p+1]) with packed FMAs - fr2 holds the
+// eight weights of its rows, each duplicated into both halves - and the four row groups are added by two
+// shuffle steps.  Returns the sums of columns 2p and 2p + 1 (valid in every lane).
+__device__ __forceinline__ float2 pass2_chunk(const uint32_t (&v)[16], float2 *tile, int lane, const float2 (&fr2)[8])
 {
 #pragma unroll
-    for (int cidx = 0; cidx < 16; ++cidx) tbuf[cidx * 36 + lane] = __uint_as_float(v[cidx]);
+    for (int pidx = 0; pidx < 8; ++pidx)
+        tile[pidx * kTcTbufStride + lane] = make_float2(__uint_as_float(v[2 * pidx]), __uint_as_float(v[2 * pidx + 1]));
     __syncwarp();
-    const float *src = tbuf + (lane & 15) * 36 + (lane & 16);
-    float2 acc[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+    const float4 *src = reinterpret_cast<const float4 *>(tile + (lane & 7) * kTcTbufStride + (lane >> 3) * 8);
+    float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
 #pragma unroll
     for (int k4 = 0; k4 < 4; ++k4) {
-        const float4 t = *reinterpret_cast<const float4 *>(src + 4 * k4);
-        acc[0] = __ffma2_rn(fr2[2 * k4], make_float2(t.x, t.y), acc[0]);
-        acc[1] = __ffma2_rn(fr2[2 * k4 + 1], make_float2(t.z, t.w), acc[1]);
+        const float4 t = src[k4];  // rows 8g + 2 k4 and 8g + 2 k4 + 1 of the pair
+        acc0 = __ffma2_rn(fr2[2 * k4], make_float2(t.x, t.y), acc0);
+        acc1 = __ffma2_rn(fr2[2 * k4 + 1], make_float2(t.z, t.w), acc1);
     }
     __syncwarp();
-    const float2 a = __fadd2_rn(acc[0], acc[1]);
-    const float part = a.x + a.y;
-    return part + __shfl_xor_sync(0xffffffffu, part, 16);
+    float2 a = __fadd2_rn(acc0, acc1);
+    a = __fadd2_rn(a, make_float2(__shfl_xor_sync(0xffffffffu, a.x, 8), __shfl_xor_sync(0xffffffffu, a.y, 8)));
+    a = __fadd2_rn(a, make_float2(__shfl_xor_sync(0xffffffffu, a.x, 16), __shfl_xor_sync(0xffffffffu, a.y, 16)));
+    return a;
 }
 
 // Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128
@@ -319,8 +327,8 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr)
     return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
            ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
 }
-// Instruction descriptor: D = fp32, A = B = bf16, both K-major, M = 128, N = 256.
-constexpr uint32_t kTcIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((256u >> 3) << 17) | ((128u >> 4) << 24);
+// Instruction descriptor: D = fp32, A = B = bf16, both K-major, M = 128, N = 128 (one column half).
+constexpr uint32_t kTcIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 
 // ------------------------------------------------------------------ the kernel
 __global__ void __launch_bounds__(kTcThreads, 1)
@@ -341,9 +349,12 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar(kBarFull + b), 1);
             mbar_init(bar(kBarEmpty + b), 1);
-            mbar_init(bar(kBarSFull + b), 1);
-            mbar_init(bar(kBarEReady + b), 256);
-            mbar_init(bar(kBarTEmpty + b), 256);
+            mbar_init(bar(kBarFReady + b), 128);
+            for (int h = 0; h < 2; ++h) {
+                mbar_init(bar(kBarSFull + 2 * b + h), 1);
+                mbar_init(bar(kBarEReady + 2 * b + h), 128);
+                mbar_init(bar(kBarTEmpty + 2 * b + h), 128);
+            }
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -383,17 +394,19 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
             for (int task = blockIdx.x; task < prm.tasks; task += gridDim.x, ++k) {
                 const uint32_t b = k & 1, ph = (k >> 1) & 1;
                 mbar_wait(bar(kBarFull + b), ph, ab, prm.status);
-                mbar_wait(bar(kBarTEmpty + b), ph ^ 1, ab, prm.status);
-                tc_fence_after();
                 const uint32_t qa = base + kTcOffStage + b * kTcStageBytes, kb = qa + kTcQBytes;
+                for (uint32_t h = 0; h < 2; ++h) {
+                    mbar_wait(bar(kBarTEmpty + 2 * b + h), ph ^ 1, ab, prm.status);
+                    tc_fence_after();
 #pragma unroll
-                for (int ks = 0; ks < kTcD / 16; ++ks) {
-                    const uint32_t blk = ks >> 2, off = (ks & 3) * 32;
-                    tc_mma_bf16(tmem + b * kTcSlab, smem_desc_sw128(qa + blk * (kTcQBytes / 2) + off),
-                                smem_desc_sw128(kb + blk * (kTcKBytes / 2) + off), kTcIdesc, ks > 0 ? 1u : 0u);
+                    for (int ks = 0; ks < kTcD / 16; ++ks) {
+                        const uint32_t blk = ks >> 2, off = (ks & 3) * 32;
+                        tc_mma_bf16(tmem + b * kTcSlab + h * 128, smem_desc_sw128(qa + blk * (kTcQBytes / 2) + off),
+                                    smem_desc_sw128(kb + blk * (kTcKBytes / 2) + h * (128 * 128) + off), kTcIdesc, ks > 0 ? 1u : 0u);
+                    }
+                    tc_commit(bar(kBarSFull + 2 * b + h));   // this half's logits are complete
                 }
-                tc_commit(bar(kBarEmpty + b));   // the stage may be refilled once these MMAs have read it
-                tc_commit(bar(kBarSFull + b));   // the logits are complete
+                tc_commit(bar(kBarEmpty + b));               // the stage may be refilled once the MMAs have read it
             }
         }
         __syncwarp();
@@ -410,7 +423,7 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
             const int nvalid = min(kTcSlab, prm.N - slab * kTcSlab);
             const uint32_t b = k & 1, ph = (k >> 1) & 1;
             const uint32_t trow = tmem + ((uint32_t)(q * 32) << 16) + b * kTcSlab + half * 128;
-            mbar_wait(bar(kBarSFull + b), ph, ab, prm.status);
+            mbar_wait(bar(kBarSFull + 2 * b + half), ph, ab, prm.status);
             tc_fence_after();
             float mxc, sum;
             if (nvalid == kTcSlab) pass1_row<true>(trow, half * 128, nvalid, c, mxc, sum);
@@ -418,7 +431,7 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
             // the reference of the stored e values (pass 2 needs it) and this half's sum
             halfst[(b * 2 + half) * kTcRows + row] = make_float2(mxc, sum);
             tc_fence_before();
-            mbar_arrive(bar(kBarEReady + b));
+            mbar_arrive(bar(kBarEReady + 2 * b + half));
             group_bar_sync<1>();
             if (half == 0) {  // merge the two halves, publish the slab's statistics of this row
                 const float2 h0 = halfst[(b * 2) * kTcRows + row], h1 = halfst[(b * 2 + 1) * kTcRows + row];
@@ -427,18 +440,15 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                 st_gpu_f32x2(&prm.stats[((size_t)item * tasks_per_item + slab) * kTcRows + row], m, l * prm.sign);
             }
         }
-    } else {
+    } else if (warp < 18) {
         // ---------------------------------------------------------------- pass 2 (256 threads)
         const int q = warp & 3;
         const int w = warp - 10;                // 0..7
         const int half = w >> 2;
-        const int row = q * 32 + lane;
         const int gt = threadIdx.x - 320;       // 0..255 within the group
-        float *tbuf = reinterpret_cast<float *>(gbase + kTcOffTbuf) + w * (16 * 36);
+        float2 *tile = reinterpret_cast<float2 *>(gbase + kTcOffTbuf) + w * (8 * kTcTbufStride);
         float *colpart = reinterpret_cast<float *>(gbase + kTcOffColpart);
-        const float2 *halfst = reinterpret_cast<const float2 *>(gbase + kTcOffHalf);
-        float *frow = reinterpret_cast<float *>(gbase + kTcOffFrow) + w * 32;
-        const float sgn = prm.sign;
+        const float *fbuf = reinterpret_cast<const float *>(gbase + kTcOffFbuf);
         uint32_t k = 0;
         for (int task = blockIdx.x; task < prm.tasks; task += gridDim.x, ++k) {
             const int item = task / tasks_per_item, slab = task - item * tasks_per_item;
@@ -446,8 +456,60 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
             const int nvalid = min(kTcSlab, prm.N - slab * kTcSlab);
             const uint32_t b = k & 1, ph = (k >> 1) & 1;
             const uint32_t trow = tmem + ((uint32_t)(q * 32) << 16) + b * kTcSlab + half * 128;
-            mbar_wait(bar(kBarEReady + b), ph, ab, prm.status);
+            mbar_wait(bar(kBarFReady + b), ph, ab, prm.status);
+            mbar_wait(bar(kBarEReady + 2 * b + half), ph, ab, prm.status);
             tc_fence_after();
+            float2 fr2[8];  // the weights of the 8 rows this lane sums over, duplicated for the packed FMAs
+            {
+                const float *fsrc = fbuf + (b * 2 + half) * kTcRows + q * 32 + (lane >> 3) * 8;
+                const float4 f0 = *reinterpret_cast<const float4 *>(fsrc), f1 = *reinterpret_cast<const float4 *>(fsrc + 4);
+                fr2[0] = make_float2(f0.x, f0.x); fr2[1] = make_float2(f0.y, f0.y);
+                fr2[2] = make_float2(f0.z, f0.z); fr2[3] = make_float2(f0.w, f0.w);
+                fr2[4] = make_float2(f1.x, f1.x); fr2[5] = make_float2(f1.y, f1.y);
+                fr2[6] = make_float2(f1.z, f1.z); fr2[7] = make_float2(f1.w, f1.w);
+            }
+            // ---- weighted column sums over this warp's 32 rows, 16 columns at a time
+            {
+                float2 *cp2 = reinterpret_cast<float2 *>(colpart + q * kTcSlab + half * 128);
+                uint32_t va[16], vb[16];
+                tmem_ld16(trow, va);
+#pragma unroll 1
+                for (int ch = 0; ch < 8; ch += 2) {
+                    tmem_wait_ld16(va);
+                    tmem_ld16(trow + (ch + 1) * 16, vb);
+                    float2 u = pass2_chunk(va, tile, lane, fr2);
+                    if (lane < 8) cp2[ch * 8 + lane] = u;
+                    tmem_wait_ld16(vb);
+                    if (ch + 2 < 8) tmem_ld16(trow + (ch + 2) * 16, va);
+                    u = pass2_chunk(vb, tile, lane, fr2);
+                    if (lane < 8) cp2[(ch + 1) * 8 + lane] = u;
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(bar(kBarTEmpty + 2 * b + half));   // this half may be overwritten by the task after next
+
+            // ---- add the four row quarters, store this task's scores
+            group_bar_sync<2>();
+            if (gt < nvalid) {
+                float *out = prm.scores + (size_t)mt * prm.part_stride + (size_t)unit * prm.N + slab * kTcSlab;
+                out[gt] = (colpart[gt] + colpart[kTcSlab + gt]) + (colpart[2 * kTcSlab + gt] + colpart[3 * kTcSlab + gt]);
+            }
+            group_bar_sync<2>();                // colpart is rewritten by the next task
+        }
+    } else {
+        // ---------------------------------------------------------------- combine (128 threads, one per query row)
+        const int row = threadIdx.x - 576;
+        const float2 *halfst = reinterpret_cast<const float2 *>(gbase + kTcOffHalf);
+        float *fbuf = reinterpret_cast<float *>(gbase + kTcOffFbuf);
+        const float sgn = prm.sign;
+        uint32_t k = 0;
+        for (int task = blockIdx.x; task < prm.tasks; task += gridDim.x, ++k) {
+            const int item = task / tasks_per_item;
+            const int mt = item % prm.mtiles;
+            const uint32_t b = k & 1, ph = (k >> 1) & 1;
+            mbar_wait(bar(kBarEReady + 2 * b), ph, ab, prm.status);
+            mbar_wait(bar(kBarEReady + 2 * b + 1), ph, ab, prm.status);
+            const float mine0 = halfst[(b * 2) * kTcRows + row].x, mine1 = halfst[(b * 2 + 1) * kTcRows + row].x;
 
             // ---- this row's statistics of every slab of the item; re-read until all carry this launch's mark
             const float2 *st = prm.stats + (size_t)item * tasks_per_item * kTcRows + row;
@@ -463,7 +525,7 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                         sv[s] = (s0 + s < tasks_per_item) ? ld_gpu_f32x2(&st[(size_t)(s0 + s) * kTcRows]) : make_float2(-INFINITY, sgn);
                         fresh = fresh && (sv[s].y * sgn > 0.f);
                     }
-                    if (!fresh && ((++tries > kTcSpinLimit / 64) || *ab)) {
+                    if (!fresh && ((++tries > kTcSpinLimit) || *ab)) {
                         if (!*ab) {
                             *ab = 1;
                             set_status(prm.status, kStatusTimeout);
@@ -481,41 +543,10 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                 m = mb;
             }
             const bool row_valid = mt * kTcRows + row < prm.M;
-            const float mine = halfst[(b * 2 + half) * kTcRows + row].x;
-            const float f = (row_valid && mine != -INFINITY) ? ex2(mine - m) / l : 0.f;
-            frow[lane] = f;
-            __syncwarp();
-            float2 fr2[8];  // the weights of the 16 rows this lane sums over
-#pragma unroll
-            for (int i = 0; i < 8; ++i) fr2[i] = *reinterpret_cast<const float2 *>(frow + (lane & 16) + 2 * i);
-            __syncwarp();
-
-            // ---- weighted column sums over this warp's 32 rows, 16 columns at a time
-            {
-                uint32_t va[16], vb[16];
-                tmem_ld16(trow, va);
-#pragma unroll 1
-                for (int ch = 0; ch < 8; ch += 2) {
-                    tmem_wait_ld16(va);
-                    tmem_ld16(trow + (ch + 1) * 16, vb);
-                    float u = pass2_chunk(va, tbuf, lane, fr2);
-                    if (lane < 16) colpart[q * kTcSlab + half * 128 + ch * 16 + lane] = u;
-                    tmem_wait_ld16(vb);
-                    if (ch + 2 < 8) tmem_ld16(trow + (ch + 2) * 16, va);
-                    u = pass2_chunk(vb, tbuf, lane, fr2);
-                    if (lane < 16) colpart[q * kTcSlab + half * 128 + (ch + 1) * 16 + lane] = u;
-                }
-            }
-            tc_fence_before();
-            mbar_arrive(bar(kBarTEmpty + b));   // the buffer may be overwritten by the task after next
-
-            // ---- add the four row quarters, store this task's scores
-            group_bar_sync<2>();
-            if (gt < nvalid) {
-                float *out = prm.scores + (size_t)mt * prm.part_stride + (size_t)unit * prm.N + slab * kTcSlab;
-                out[gt] = (colpart[gt] + colpart[kTcSlab + gt]) + (colpart[2 * kTcSlab + gt] + colpart[3 * kTcSlab + gt]);
-            }
-            group_bar_sync<2>();                // colpart is rewritten by the next task
+            const float inv_l = row_valid ? 1.f / l : 0.f;
+            fbuf[(b * 2) * kTcRows + row] = ex2(mine0 - m) * inv_l;
+            fbuf[(b * 2 + 1) * kTcRows + row] = (mine1 == -INFINITY) ? 0.f : ex2(mine1 - m) * inv_l;
+            mbar_arrive(bar(kBarFReady + b));
         }
     }
 
