@@ -10,19 +10,24 @@
 //   TMA      Q tile (128 x 128 bf16) and the slab's keys (256 x 128 bf16) land in
 //            shared memory in the 128-byte-swizzled K-major layout (2 stages);
 //   tcgen05  S = Q K^T (128 x 256 fp32) accumulates in one of two 256-column tensor
-//            memory buffers: the logits never leave the SM;
-//   pass 1   (warps 2-9, two threads per query row, 128 columns each) maximum,
-//            e = 2^(x - max) written back over the logits, sum; the row's slab
-//            statistics (max, sum) go to a small global array, one 8-byte store per
-//            row whose sum carries the launch's sign as a "fresh" mark;
-//   combine  (warps 18-21, one thread per query row) reads the row's statistics of
-//            all slabs of the item, re-reading until every one is fresh - normally
-//            they are, as the CTA has meanwhile started pass 1 of its next task -
-//            and turns them into the row's global maximum m, denominator l and the
-//            weights 2^(max - m) / l of the stored e values;
-//   pass 2   (warps 10-17) u_j = sum_i e_ij 2^(max_i - m_i) / l_i as a weighted
-//            column sum (per-warp shared-memory transpose, then across the four row
-//            quarters), stored: 256 floats per task.
+//            memory buffers, one 128-column half at a time: the logits never leave
+//            the SM;
+//   pass 1   (16 epilogue warps; a thread owns one query row x 64 columns, 32 in each
+//            half of the buffer) maximum, e = 2^(x - max) written back over the
+//            logits, sum;
+//   combine  (4 warps, one thread per query row) merges the four (max, sum) pairs of
+//            its row into the slab's statistics and publishes them with one 8-byte
+//            store whose sum carries the launch's sign as a "fresh" mark; then reads
+//            the row's statistics of all slabs of the item, re-reading until every
+//            one is fresh, and turns them into the row's global maximum m, its
+//            denominator l and the weights 2^(max - m) / l of the stored e values;
+//   pass 2   (the same 16 warps, one task behind: after pass 1 of task t+1 they
+//            finish task t, whose weights have arrived meanwhile)
+//            u_j = sum_i e_ij 2^(max_i - m_i) / l_i as a weighted column sum: the
+//            16x256b tensor-memory load shape hands every thread four rows of a
+//            column pair, so the sum over a warp's 32 rows is four packed FMAs plus
+//            a three-step exchange between lanes; the four row quarters are added
+//            through shared memory and stored: 256 floats per task.
 // The two 128-column halves of a buffer are handed over separately (MMA -> pass 1,
 // pass 2 -> MMA), so the tensor core refills one half while the other is still read.
 //
@@ -42,7 +47,7 @@
 
 namespace ipotk {
 
-constexpr int kTcThreads = 704;      // warp 0: TMA, 1: MMA + TMEM owner, 2-9: pass 1, 10-17: pass 2, 18-21: combine
+constexpr int kTcThreads = 704;      // warp 0: TMA, 1: MMA + TMEM owner, 2-17: pass 1 / pass 2, 18-21: combine
 constexpr int kTcRows = 128;         // query rows per item (TMEM lanes)
 constexpr int kTcSlab = 256;         // keys per task (TMEM columns per buffer)
 constexpr int kTcD = 128;
@@ -53,16 +58,14 @@ constexpr uint32_t kTcSpinLimit = 1u << 18;                  // try_wait / poll 
 
 // shared-memory carve-up (bytes from the 1024-aligned base)
 constexpr uint32_t kTcOffStage = 0;                                        // [2] { Q, K }
-constexpr uint32_t kTcTbufStride = 34;                                     // float2 per column pair (32 rows + pad)
-constexpr uint32_t kTcOffTbuf = 2 * kTcStageBytes;                         // [8 warps][8 pairs][34] float2
-constexpr uint32_t kTcOffColpart = kTcOffTbuf + 8 * 8 * kTcTbufStride * 8; // [4][256] float
-constexpr uint32_t kTcOffHalf = kTcOffColpart + 4 * kTcSlab * 4;           // [2 buffers][2 halves][128] float2
-constexpr uint32_t kTcOffFbuf = kTcOffHalf + 2 * 2 * kTcRows * 8;          // [2 buffers][2 halves][128] float
-constexpr uint32_t kTcOffBar = kTcOffFbuf + 2 * 2 * kTcRows * 4;
+constexpr uint32_t kTcOffColpart = 2 * kTcStageBytes;                      // [4][256] float
+constexpr uint32_t kTcOffTstat = kTcOffColpart + 4 * kTcSlab * 4;          // [2 buffers][4 column quarters][128] float2
+constexpr uint32_t kTcOffFbuf = kTcOffTstat + 2 * 4 * kTcRows * 8;         // [2 buffers][4 column quarters][128] float
+constexpr uint32_t kTcOffBar = kTcOffFbuf + 2 * 4 * kTcRows * 4;
 constexpr uint32_t kTcSmemBytes = kTcOffBar + 256 + 1024;                  // + alignment slack
 
-// barriers: per stage Full, Empty, FReady; per (buffer, half) SFull, EReady, TEmpty at index 2 * buffer + half
-enum { kBarFull = 0, kBarEmpty = 2, kBarFReady = 4, kBarSFull = 6, kBarEReady = 10, kBarTEmpty = 14, kBarCount = 18 };
+// barriers: per stage Full, Empty, EReady, FReady; per (buffer, half) SFull, TEmpty at index 2 * buffer + half
+enum { kBarFull = 0, kBarEmpty = 2, kBarEReady = 4, kBarFReady = 6, kBarSFull = 8, kBarTEmpty = 12, kBarCount = 16 };
 
 struct TcParams {
     float *scores;        // partial array p (query rows 128p ...) at scores + p * part_stride, unit stride N
@@ -146,10 +149,12 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32])
           "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
         : "r"(taddr) : "memory");
 }
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16])
+// 16 TMEM lanes x 32 fp32 columns in the 16x256b shape: for each block j of 8 columns, thread t of the warp
+// receives v[4j], v[4j+1] = lane t/4, columns 8j + 2(t%4), +1 and v[4j+2], v[4j+3] = lane t/4 + 8, same columns.
+__device__ __forceinline__ void tmem_ld_16x256b_x4(uint32_t taddr, uint32_t (&v)[16])
 {
     asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "tcgen05.ld.sync.aligned.16x256b.x4.b32 "
         "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
         : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
           "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
@@ -190,9 +195,9 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 template <int kId>
-__device__ __forceinline__ void group_bar_sync()  // 256-thread named barrier of one epilogue group
+__device__ __forceinline__ void group_bar_sync()  // named barrier of the 512 epilogue threads
 {
-    asm volatile("bar.sync %0, 256;" ::"n"(kId) : "memory");
+    asm volatile("bar.sync %0, 512;" ::"n"(kId) : "memory");
 }
 // The slab statistics are exchanged between CTAs with single 8-byte relaxed accesses at gpu scope:
 // one store publishes (max, marked sum) together, and a reader sees either the old or the new pair.
@@ -255,69 +260,72 @@ __device__ __forceinline__ void chunk_exp(uint32_t (&v)[32], int col0, int nvali
     }
 }
 
-// Pass 1 for one query row over 128 columns starting at col0: returns their maximum (log2 units) and
-// sum of e = 2^(x - max), and leaves e in tensor memory.  TMEM loads run one 32-column chunk ahead of
-// the arithmetic.  With no valid column the maximum is -inf, the sum 0 and zeros are stored.
-template <bool kFull>
-__device__ __forceinline__ void pass1_row(uint32_t trow, int col0, int nvalid, float c, float &mxc_out, float &sum_out)
+// Pass 1 for one query row over its 64 columns: 32 at t0 (slab columns from col0) and 32 at t1 (from col1).
+// Returns their maximum (log2 units) and the sum of e = 2^(x - max), and leaves e in tensor memory.  With
+// no valid column the maximum is -inf, the sum 0 and zeros are stored.  `wait_second` is called before the
+// second chunk is first touched (its half of the buffer is completed later than the first).
+template <bool kFull, typename WaitSecond>
+__device__ __forceinline__ void pass1_row(uint32_t t0, uint32_t t1, int col0, int col1, int nvalid, float c,
+                                          WaitSecond wait_second, float &mxc_out, float &sum_out)
 {
-    uint32_t va[32], vb[32];
+    uint32_t v[32];
     float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-    tmem_ld32(trow, va);
-#pragma unroll 1
-    for (int ch = 0; ch < 4; ch += 2) {
-        tmem_wait_ld(va);
-        tmem_ld32(trow + (ch + 1) * 32, vb);
-        chunk_max<kFull>(va, col0 + ch * 32, nvalid, mx);
-        tmem_wait_ld(vb);
-        if (ch + 2 < 4) tmem_ld32(trow + (ch + 2) * 32, va);
-        chunk_max<kFull>(vb, col0 + (ch + 1) * 32, nvalid, mx);
-    }
+    tmem_ld32(t0, v);
+    tmem_wait_ld(v);
+    chunk_max<kFull>(v, col0, nvalid, mx);
+    wait_second();
+    tmem_ld32(t1, v);
+    tmem_wait_ld(v);
+    chunk_max<kFull>(v, col1, nvalid, mx);
     const float mxr = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
     const float mxc = (mxr == -INFINITY) ? 0.f : mxr * c;
     float2 sum[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-    tmem_ld32(trow, va);
-#pragma unroll 1
-    for (int ch = 0; ch < 4; ch += 2) {
-        tmem_wait_ld(va);
-        tmem_ld32(trow + (ch + 1) * 32, vb);
-        chunk_exp<kFull>(va, col0 + ch * 32, nvalid, c, mxc, sum);
-        tmem_st32(trow + ch * 32, va);
-        tmem_wait_ld(vb);
-        if (ch + 2 < 4) tmem_ld32(trow + (ch + 2) * 32, va);
-        chunk_exp<kFull>(vb, col0 + (ch + 1) * 32, nvalid, c, mxc, sum);
-        tmem_st32(trow + (ch + 1) * 32, vb);
-    }
+    chunk_exp<kFull>(v, col1, nvalid, c, mxc, sum);  // the second chunk is still in registers
+    tmem_st32(t1, v);
+    tmem_ld32(t0, v);
+    tmem_wait_ld(v);
+    chunk_exp<kFull>(v, col0, nvalid, c, mxc, sum);
+    tmem_st32(t0, v);
     tmem_wait_st();
     const float2 s01 = __fadd2_rn(sum[0], sum[1]), s23 = __fadd2_rn(sum[2], sum[3]);
     mxc_out = (mxr == -INFINITY) ? -INFINITY : mxc;
     sum_out = (s01.x + s01.y) + (s23.x + s23.y);
 }
 
-// One 16-column chunk of pass 2 for one warp (32 rows).  The chunk is transposed through the warp's
-// shared-memory tile as 8 column pairs: tile[pair][row] (float2, row stride 34).  Lane (g, p) = (lane / 8,
-// lane % 8) then forms sum_{r in 8g..8g+7} f_r (e[r][2p], e[r][2p+1]) with packed FMAs - fr2 holds the
-// eight weights of its rows, each duplicated into both halves - and the four row groups are added by two
-// shuffle steps.  Returns the sums of columns 2p and 2p + 1 (valid in every lane).
-__device__ __forceinline__ float2 pass2_chunk(const uint32_t (&v)[16], float2 *tile, int lane, const float2 (&fr2)[8])
+// Pass 2 for one warp over 32 rows x 32 columns: a[] and b[] are the 16x256b loads of the warp's TMEM lanes
+// 0..15 and 16..31, fr2[i] the weight of row lane/4 + 8i duplicated into both halves.  On exit
+// x[2j + h] = sum over this thread's four rows of f_r e[r][8j + 2(lane%4) + h].
+__device__ __forceinline__ void pass2_rows(const uint32_t (&a)[16], const uint32_t (&b)[16], const float2 (&fr2)[4], float (&x)[8])
 {
 #pragma unroll
-    for (int pidx = 0; pidx < 8; ++pidx)
-        tile[pidx * kTcTbufStride + lane] = make_float2(__uint_as_float(v[2 * pidx]), __uint_as_float(v[2 * pidx + 1]));
-    __syncwarp();
-    const float4 *src = reinterpret_cast<const float4 *>(tile + (lane & 7) * kTcTbufStride + (lane >> 3) * 8);
-    float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
-#pragma unroll
-    for (int k4 = 0; k4 < 4; ++k4) {
-        const float4 t = src[k4];  // rows 8g + 2 k4 and 8g + 2 k4 + 1 of the pair
-        acc0 = __ffma2_rn(fr2[2 * k4], make_float2(t.x, t.y), acc0);
-        acc1 = __ffma2_rn(fr2[2 * k4 + 1], make_float2(t.z, t.w), acc1);
+    for (int j = 0; j < 4; ++j) {
+        float2 s = __ffma2_rn(fr2[0], make_float2(__uint_as_float(a[4 * j]), __uint_as_float(a[4 * j + 1])), make_float2(0.f, 0.f));
+        s = __ffma2_rn(fr2[1], make_float2(__uint_as_float(a[4 * j + 2]), __uint_as_float(a[4 * j + 3])), s);
+        s = __ffma2_rn(fr2[2], make_float2(__uint_as_float(b[4 * j]), __uint_as_float(b[4 * j + 1])), s);
+        s = __ffma2_rn(fr2[3], make_float2(__uint_as_float(b[4 * j + 2]), __uint_as_float(b[4 * j + 3])), s);
+        x[2 * j] = s.x;
+        x[2 * j + 1] = s.y;
     }
-    __syncwarp();
-    float2 a = __fadd2_rn(acc0, acc1);
-    a = __fadd2_rn(a, make_float2(__shfl_xor_sync(0xffffffffu, a.x, 8), __shfl_xor_sync(0xffffffffu, a.y, 8)));
-    a = __fadd2_rn(a, make_float2(__shfl_xor_sync(0xffffffffu, a.x, 16), __shfl_xor_sync(0xffffffffu, a.y, 16)));
-    return a;
+}
+
+// Adds the partial sums of the eight lanes that share lane % 4: on entry lane (g, p) = (lane / 4, lane % 4) holds
+// x[2c + h] = its partial of column 8c + 2p + h (c < 4, h < 2); on exit it holds the complete sum of column
+// 8 (g / 2) + 2p + (g % 2).  Three exchange steps, each halving the values a lane carries.
+__device__ __forceinline__ float pass2_reduce(float (&x)[8], int lane)
+{
+    const bool up4 = lane & 16, up2 = lane & 8, up1 = lane & 4;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {  // g bit 2 picks x[4..7] or x[0..3]
+        const float keep = up4 ? x[i + 4] : x[i], give = up4 ? x[i] : x[i + 4];
+        x[i] = keep + __shfl_xor_sync(0xffffffffu, give, 16);
+    }
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {  // g bit 1 picks x[2..3] or x[0..1]
+        const float keep = up2 ? x[i + 2] : x[i], give = up2 ? x[i] : x[i + 2];
+        x[i] = keep + __shfl_xor_sync(0xffffffffu, give, 8);
+    }
+    const float keep = up1 ? x[1] : x[0], give = up1 ? x[0] : x[1];
+    return keep + __shfl_xor_sync(0xffffffffu, give, 4);
 }
 
 // Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128
@@ -349,11 +357,11 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar(kBarFull + b), 1);
             mbar_init(bar(kBarEmpty + b), 1);
+            mbar_init(bar(kBarEReady + b), 512);
             mbar_init(bar(kBarFReady + b), 128);
             for (int h = 0; h < 2; ++h) {
                 mbar_init(bar(kBarSFull + 2 * b + h), 1);
-                mbar_init(bar(kBarEReady + 2 * b + h), 128);
-                mbar_init(bar(kBarTEmpty + 2 * b + h), 128);
+                mbar_init(bar(kBarTEmpty + 2 * b + h), 512);
             }
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -410,106 +418,101 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
             }
         }
         __syncwarp();
-    } else if (warp < 10) {
-        // ---------------------------------------------------------------- pass 1 (256 threads: row x column half)
-        const int q = warp & 3;                 // TMEM lane quarter this warp may touch
-        const int half = (warp - 2) >> 2;       // which 128 columns of the slab
-        const int row = q * 32 + lane;
-        float2 *halfst = reinterpret_cast<float2 *>(gbase + kTcOffHalf);
-        const float c = prm.scale_log2e;
-        uint32_t k = 0;
-        for (int task = blockIdx.x; task < prm.tasks; task += gridDim.x, ++k) {
-            const int item = task / tasks_per_item, slab = task - item * tasks_per_item;
-            const int nvalid = min(kTcSlab, prm.N - slab * kTcSlab);
-            const uint32_t b = k & 1, ph = (k >> 1) & 1;
-            const uint32_t trow = tmem + ((uint32_t)(q * 32) << 16) + b * kTcSlab + half * 128;
-            mbar_wait(bar(kBarSFull + 2 * b + half), ph, ab, prm.status);
-            tc_fence_after();
-            float mxc, sum;
-            if (nvalid == kTcSlab) pass1_row<true>(trow, half * 128, nvalid, c, mxc, sum);
-            else pass1_row<false>(trow, half * 128, nvalid, c, mxc, sum);
-            // the reference of the stored e values (pass 2 needs it) and this half's sum
-            halfst[(b * 2 + half) * kTcRows + row] = make_float2(mxc, sum);
-            tc_fence_before();
-            mbar_arrive(bar(kBarEReady + 2 * b + half));
-            group_bar_sync<1>();
-            if (half == 0) {  // merge the two halves, publish the slab's statistics of this row
-                const float2 h0 = halfst[(b * 2) * kTcRows + row], h1 = halfst[(b * 2 + 1) * kTcRows + row];
-                const float m = fmaxf(h0.x, h1.x);  // half 0 always holds a valid key
-                const float l = h0.y * ex2(h0.x - m) + (h1.x == -INFINITY ? 0.f : h1.y * ex2(h1.x - m));
-                st_gpu_f32x2(&prm.stats[((size_t)item * tasks_per_item + slab) * kTcRows + row], m, l * prm.sign);
-            }
-        }
     } else if (warp < 18) {
-        // ---------------------------------------------------------------- pass 2 (256 threads)
-        const int q = warp & 3;
-        const int w = warp - 10;                // 0..7
-        const int half = w >> 2;
-        const int gt = threadIdx.x - 320;       // 0..255 within the group
-        float2 *tile = reinterpret_cast<float2 *>(gbase + kTcOffTbuf) + w * (8 * kTcTbufStride);
-        float *colpart = reinterpret_cast<float *>(gbase + kTcOffColpart);
+        // ---------------------------------------------------------------- pass 1 / pass 2 (512 threads)
+        const int q = warp & 3;                 // TMEM lane quarter this warp may touch
+        const int w = warp - 2;                 // 0..15
+        const int cq = w >> 2;                  // this warp's columns: [32 cq, 32 cq + 32) of each buffer half
+        const int row = q * 32 + lane;
+        const int gt = threadIdx.x - 64;        // 0..511 within the group
+        float2 *tstat = reinterpret_cast<float2 *>(gbase + kTcOffTstat);
         const float *fbuf = reinterpret_cast<const float *>(gbase + kTcOffFbuf);
-        uint32_t k = 0;
-        for (int task = blockIdx.x; task < prm.tasks; task += gridDim.x, ++k) {
-            const int item = task / tasks_per_item, slab = task - item * tasks_per_item;
-            const int unit = item / prm.mtiles, mt = item - unit * prm.mtiles;
-            const int nvalid = min(kTcSlab, prm.N - slab * kTcSlab);
-            const uint32_t b = k & 1, ph = (k >> 1) & 1;
-            const uint32_t trow = tmem + ((uint32_t)(q * 32) << 16) + b * kTcSlab + half * 128;
-            mbar_wait(bar(kBarFReady + b), ph, ab, prm.status);
-            mbar_wait(bar(kBarEReady + 2 * b + half), ph, ab, prm.status);
-            tc_fence_after();
-            float2 fr2[8];  // the weights of the 8 rows this lane sums over, duplicated for the packed FMAs
-            {
-                const float *fsrc = fbuf + (b * 2 + half) * kTcRows + q * 32 + (lane >> 3) * 8;
-                const float4 f0 = *reinterpret_cast<const float4 *>(fsrc), f1 = *reinterpret_cast<const float4 *>(fsrc + 4);
-                fr2[0] = make_float2(f0.x, f0.x); fr2[1] = make_float2(f0.y, f0.y);
-                fr2[2] = make_float2(f0.z, f0.z); fr2[3] = make_float2(f0.w, f0.w);
-                fr2[4] = make_float2(f1.x, f1.x); fr2[5] = make_float2(f1.y, f1.y);
-                fr2[6] = make_float2(f1.z, f1.z); fr2[7] = make_float2(f1.w, f1.w);
+        float *colpart = reinterpret_cast<float *>(gbase + kTcOffColpart);
+        const float c = prm.scale_log2e;
+        const int n_local = (prm.tasks - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+        for (int k = 0; k <= n_local; ++k) {
+            if (k < n_local) {
+                // ---- pass 1 of local task k
+                const int task = blockIdx.x + k * gridDim.x;
+                const int slab = task % tasks_per_item;
+                const int nvalid = min(kTcSlab, prm.N - slab * kTcSlab);
+                const uint32_t b = k & 1, ph = (k >> 1) & 1;
+                const uint32_t t0 = tmem + ((uint32_t)(q * 32) << 16) + b * kTcSlab + cq * 32, t1 = t0 + 128;
+                mbar_wait(bar(kBarSFull + 2 * b), ph, ab, prm.status);
+                tc_fence_after();
+                auto wait_second = [&]() {
+                    mbar_wait(bar(kBarSFull + 2 * b + 1), ph, ab, prm.status);
+                    tc_fence_after();
+                };
+                float mxc, sum;
+                if (nvalid == kTcSlab) pass1_row<true>(t0, t1, cq * 32, 128 + cq * 32, nvalid, c, wait_second, mxc, sum);
+                else pass1_row<false>(t0, t1, cq * 32, 128 + cq * 32, nvalid, c, wait_second, mxc, sum);
+                tstat[(b * 4 + cq) * kTcRows + row] = make_float2(mxc, sum);
+                tc_fence_before();  // pass 2 reads these TMEM words from other lanes of the warp
+                mbar_arrive(bar(kBarEReady + b));
             }
-            // ---- weighted column sums over this warp's 32 rows, 16 columns at a time
-            {
-                float2 *cp2 = reinterpret_cast<float2 *>(colpart + q * kTcSlab + half * 128);
-                uint32_t va[16], vb[16];
-                tmem_ld16(trow, va);
-#pragma unroll 1
-                for (int ch = 0; ch < 8; ch += 2) {
-                    tmem_wait_ld16(va);
-                    tmem_ld16(trow + (ch + 1) * 16, vb);
-                    float2 u = pass2_chunk(va, tile, lane, fr2);
-                    if (lane < 8) cp2[ch * 8 + lane] = u;
-                    tmem_wait_ld16(vb);
-                    if (ch + 2 < 8) tmem_ld16(trow + (ch + 2) * 16, va);
-                    u = pass2_chunk(vb, tile, lane, fr2);
-                    if (lane < 8) cp2[(ch + 1) * 8 + lane] = u;
+            if (k >= 1) {
+                // ---- pass 2 of local task k - 1
+                const int kk = k - 1;
+                const int task = blockIdx.x + kk * gridDim.x;
+                const int item = task / tasks_per_item, slab = task - item * tasks_per_item;
+                const int unit = item / prm.mtiles, mt = item - unit * prm.mtiles;
+                const int nvalid = min(kTcSlab, prm.N - slab * kTcSlab);
+                const uint32_t b = kk & 1, ph = (kk >> 1) & 1;
+                const uint32_t trow = tmem + ((uint32_t)(q * 32) << 16) + b * kTcSlab + cq * 32;
+                mbar_wait(bar(kBarFReady + b), ph, ab, prm.status);
+                tc_fence_after();
+                float2 fr2[4];  // the weights of rows lane/4 + 8i of this warp's quarter, duplicated for the packed FMAs
+                {
+                    const float *f = fbuf + (b * 4 + cq) * kTcRows + q * 32 + (lane >> 2);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) fr2[i] = make_float2(f[8 * i], f[8 * i]);
                 }
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {  // this warp's 32 columns of buffer half h
+                    uint32_t va[16], vb[16];
+                    tmem_ld_16x256b_x4(trow + h * 128, va);
+                    tmem_ld_16x256b_x4(trow + h * 128 + (16u << 16), vb);
+                    tmem_wait_ld16(va);
+                    tmem_wait_ld16(vb);
+                    tc_fence_before();
+                    mbar_arrive(bar(kBarTEmpty + 2 * b + h));   // this half may be overwritten by the task after next
+                    float x[8];
+                    pass2_rows(va, vb, fr2, x);
+                    const float u = pass2_reduce(x, lane);
+                    const int g = lane >> 2, pp = lane & 3;
+                    colpart[q * kTcSlab + h * 128 + cq * 32 + 8 * (g >> 1) + 2 * pp + (g & 1)] = u;
+                }
+                // ---- add the four row quarters, store this task's scores
+                group_bar_sync<1>();
+                if (gt < nvalid) {
+                    float *out = prm.scores + (size_t)mt * prm.part_stride + (size_t)unit * prm.N + slab * kTcSlab;
+                    out[gt] = (colpart[gt] + colpart[kTcSlab + gt]) + (colpart[2 * kTcSlab + gt] + colpart[3 * kTcSlab + gt]);
+                }
+                group_bar_sync<1>();                // colpart is rewritten by the next task
             }
-            tc_fence_before();
-            mbar_arrive(bar(kBarTEmpty + 2 * b + half));   // this half may be overwritten by the task after next
-
-            // ---- add the four row quarters, store this task's scores
-            group_bar_sync<2>();
-            if (gt < nvalid) {
-                float *out = prm.scores + (size_t)mt * prm.part_stride + (size_t)unit * prm.N + slab * kTcSlab;
-                out[gt] = (colpart[gt] + colpart[kTcSlab + gt]) + (colpart[2 * kTcSlab + gt] + colpart[3 * kTcSlab + gt]);
-            }
-            group_bar_sync<2>();                // colpart is rewritten by the next task
         }
     } else {
         // ---------------------------------------------------------------- combine (128 threads, one per query row)
         const int row = threadIdx.x - 576;
-        const float2 *halfst = reinterpret_cast<const float2 *>(gbase + kTcOffHalf);
+        const float2 *tstat = reinterpret_cast<const float2 *>(gbase + kTcOffTstat);
         float *fbuf = reinterpret_cast<float *>(gbase + kTcOffFbuf);
         const float sgn = prm.sign;
         uint32_t k = 0;
         for (int task = blockIdx.x; task < prm.tasks; task += gridDim.x, ++k) {
-            const int item = task / tasks_per_item;
+            const int item = task / tasks_per_item, slab = task - item * tasks_per_item;
             const int mt = item % prm.mtiles;
             const uint32_t b = k & 1, ph = (k >> 1) & 1;
-            mbar_wait(bar(kBarEReady + 2 * b), ph, ab, prm.status);
-            mbar_wait(bar(kBarEReady + 2 * b + 1), ph, ab, prm.status);
-            const float mine0 = halfst[(b * 2) * kTcRows + row].x, mine1 = halfst[(b * 2 + 1) * kTcRows + row].x;
+            mbar_wait(bar(kBarEReady + b), ph, ab, prm.status);
+            // ---- merge the four column quarters of the row, publish the slab's statistics
+            float2 t4[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) t4[i] = tstat[(b * 4 + i) * kTcRows + row];
+            const float ms = fmaxf(fmaxf(t4[0].x, t4[1].x), fmaxf(t4[2].x, t4[3].x));  // quarter 0 always holds a valid key
+            float ls = 0.f;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) ls += (t4[i].x == -INFINITY) ? 0.f : t4[i].y * ex2(t4[i].x - ms);
+            st_gpu_f32x2(&prm.stats[((size_t)item * tasks_per_item + slab) * kTcRows + row], ms, ls * sgn);
 
             // ---- this row's statistics of every slab of the item; re-read until all carry this launch's mark
             const float2 *st = prm.stats + (size_t)item * tasks_per_item * kTcRows + row;
@@ -532,7 +535,6 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                         }
                         break;
                     }
-                    if (!fresh) __nanosleep(100);
                 } while (!fresh);
                 float mb = m;
 #pragma unroll
@@ -544,8 +546,9 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
             }
             const bool row_valid = mt * kTcRows + row < prm.M;
             const float inv_l = row_valid ? 1.f / l : 0.f;
-            fbuf[(b * 2) * kTcRows + row] = ex2(mine0 - m) * inv_l;
-            fbuf[(b * 2 + 1) * kTcRows + row] = (mine1 == -INFINITY) ? 0.f : ex2(mine1 - m) * inv_l;
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                fbuf[(b * 4 + i) * kTcRows + row] = (t4[i].x == -INFINITY) ? 0.f : ex2(t4[i].x - m) * inv_l;
             mbar_arrive(bar(kBarFReady + b));
         }
     }
