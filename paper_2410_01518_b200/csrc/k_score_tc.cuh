@@ -12,15 +12,16 @@
 //   tcgen05  S = Q K^T (128 x 256 fp32) accumulates in one of two 256-column tensor
 //            memory buffers, one 128-column half at a time: the logits never leave
 //            the SM;
-//   pass 1   (16 epilogue warps; a thread owns one query row x 64 columns, 32 in each
-//            half of the buffer) maximum, e = 2^(x - max) written back over the
-//            logits, sum;
-//   combine  (4 warps, one thread per query row) merges the four (max, sum) pairs of
+//   pass 1   (16 epilogue warps; a thread owns one query row x two chunks of 32 columns,
+//            one in each half of the buffer) per chunk: maximum, e = 2^(x - max)
+//            written back over the logits, sum - one tensor-memory read and one
+//            write per logit;
+//   combine  (4 warps, one thread per query row) merges the eight (max, sum) pairs of
 //            its row into the slab's statistics and publishes them with one 8-byte
 //            store whose sum carries the launch's sign as a "fresh" mark; then reads
 //            the row's statistics of all slabs of the item, re-reading until every
 //            one is fresh, and turns them into the row's global maximum m, its
-//            denominator l and the weights 2^(max - m) / l of the stored e values;
+//            denominator l and the weights 2^(max_chunk - m) / l of the stored e values;
 //   pass 2   (the same 16 warps, one task behind: after pass 1 of task t+1 they
 //            finish task t, whose weights have arrived meanwhile)
 //            u_j = sum_i e_ij 2^(max_i - m_i) / l_i as a weighted column sum: the
@@ -54,14 +55,14 @@ constexpr int kTcD = 128;
 constexpr uint32_t kTcQBytes = kTcRows * kTcD * 2;           // 32 KiB
 constexpr uint32_t kTcKBytes = kTcSlab * kTcD * 2;           // 64 KiB
 constexpr uint32_t kTcStageBytes = kTcQBytes + kTcKBytes;    // 96 KiB
-constexpr uint32_t kTcSpinLimit = 1u << 18;                  // try_wait / poll rounds before giving up
+constexpr uint32_t kTcSpinLimit = 1u << 22;                  // try_wait / poll rounds before giving up
 
 // shared-memory carve-up (bytes from the 1024-aligned base)
 constexpr uint32_t kTcOffStage = 0;                                        // [2] { Q, K }
 constexpr uint32_t kTcOffColpart = 2 * kTcStageBytes;                      // [4][256] float
-constexpr uint32_t kTcOffTstat = kTcOffColpart + 4 * kTcSlab * 4;          // [2 buffers][4 column quarters][128] float2
-constexpr uint32_t kTcOffFbuf = kTcOffTstat + 2 * 4 * kTcRows * 8;         // [2 buffers][4 column quarters][128] float
-constexpr uint32_t kTcOffBar = kTcOffFbuf + 2 * 4 * kTcRows * 4;
+constexpr uint32_t kTcOffTstat = kTcOffColpart + 4 * kTcSlab * 4;          // [2 buffers][8 chunks][128] float2
+constexpr uint32_t kTcOffFbuf = kTcOffTstat + 2 * 8 * kTcRows * 8;         // [2 buffers][8 chunks][128] float
+constexpr uint32_t kTcOffBar = kTcOffFbuf + 2 * 8 * kTcRows * 4;
 constexpr uint32_t kTcSmemBytes = kTcOffBar + 256 + 1024;                  // + alignment slack
 
 // barriers: per stage Full, Empty, EReady, FReady; per (buffer, half) SFull, TEmpty at index 2 * buffer + half
@@ -97,9 +98,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity), "r"(20000u) : "memory");  // may sleep up to ~20 us per try
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
 // Bounded wait.  Once any wait of the CTA has run out, later waits return at once.
@@ -260,36 +261,24 @@ __device__ __forceinline__ void chunk_exp(uint32_t (&v)[32], int col0, int nvali
     }
 }
 
-// Pass 1 for one query row over its 64 columns: 32 at t0 (slab columns from col0) and 32 at t1 (from col1).
-// Returns their maximum (log2 units) and the sum of e = 2^(x - max), and leaves e in tensor memory.  With
-// no valid column the maximum is -inf, the sum 0 and zeros are stored.  `wait_second` is called before the
-// second chunk is first touched (its half of the buffer is completed later than the first).
-template <bool kFull, typename WaitSecond>
-__device__ __forceinline__ void pass1_row(uint32_t t0, uint32_t t1, int col0, int col1, int nvalid, float c,
-                                          WaitSecond wait_second, float &mxc_out, float &sum_out)
+// Pass 1 for one query row over one chunk of 32 columns (slab columns from col0): returns the chunk's
+// maximum (log2 units) and the sum of e = 2^(x - max), and leaves e in tensor memory.  With no valid column
+// the maximum is -inf, the sum 0 and zeros are stored.
+template <bool kFull>
+__device__ __forceinline__ float2 pass1_chunk(uint32_t taddr, int col0, int nvalid, float c)
 {
     uint32_t v[32];
     float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-    tmem_ld32(t0, v);
+    tmem_ld32(taddr, v);
     tmem_wait_ld(v);
     chunk_max<kFull>(v, col0, nvalid, mx);
-    wait_second();
-    tmem_ld32(t1, v);
-    tmem_wait_ld(v);
-    chunk_max<kFull>(v, col1, nvalid, mx);
     const float mxr = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
     const float mxc = (mxr == -INFINITY) ? 0.f : mxr * c;
     float2 sum[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-    chunk_exp<kFull>(v, col1, nvalid, c, mxc, sum);  // the second chunk is still in registers
-    tmem_st32(t1, v);
-    tmem_ld32(t0, v);
-    tmem_wait_ld(v);
     chunk_exp<kFull>(v, col0, nvalid, c, mxc, sum);
-    tmem_st32(t0, v);
-    tmem_wait_st();
+    tmem_st32(taddr, v);
     const float2 s01 = __fadd2_rn(sum[0], sum[1]), s23 = __fadd2_rn(sum[2], sum[3]);
-    mxc_out = (mxr == -INFINITY) ? -INFINITY : mxc;
-    sum_out = (s01.x + s01.y) + (s23.x + s23.y);
+    return make_float2((mxr == -INFINITY) ? -INFINITY : mxc, (s01.x + s01.y) + (s23.x + s23.y));
 }
 
 // Pass 2 for one warp over 32 rows x 32 columns: a[] and b[] are the 16x256b loads of the warp's TMEM lanes
@@ -437,17 +426,16 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                 const int slab = task % tasks_per_item;
                 const int nvalid = min(kTcSlab, prm.N - slab * kTcSlab);
                 const uint32_t b = k & 1, ph = (k >> 1) & 1;
-                const uint32_t t0 = tmem + ((uint32_t)(q * 32) << 16) + b * kTcSlab + cq * 32, t1 = t0 + 128;
-                mbar_wait(bar(kBarSFull + 2 * b), ph, ab, prm.status);
-                tc_fence_after();
-                auto wait_second = [&]() {
-                    mbar_wait(bar(kBarSFull + 2 * b + 1), ph, ab, prm.status);
+                const uint32_t t0 = tmem + ((uint32_t)(q * 32) << 16) + b * kTcSlab + cq * 32;
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    mbar_wait(bar(kBarSFull + 2 * b + h), ph, ab, prm.status);
                     tc_fence_after();
-                };
-                float mxc, sum;
-                if (nvalid == kTcSlab) pass1_row<true>(t0, t1, cq * 32, 128 + cq * 32, nvalid, c, wait_second, mxc, sum);
-                else pass1_row<false>(t0, t1, cq * 32, 128 + cq * 32, nvalid, c, wait_second, mxc, sum);
-                tstat[(b * 4 + cq) * kTcRows + row] = make_float2(mxc, sum);
+                    const float2 st = (nvalid == kTcSlab) ? pass1_chunk<true>(t0 + h * 128, h * 128 + cq * 32, nvalid, c)
+                                                          : pass1_chunk<false>(t0 + h * 128, h * 128 + cq * 32, nvalid, c);
+                    tstat[(b * 8 + h * 4 + cq) * kTcRows + row] = st;
+                }
+                tmem_wait_st();
                 tc_fence_before();  // pass 2 reads these TMEM words from other lanes of the warp
                 mbar_arrive(bar(kBarEReady + b));
             }
@@ -462,14 +450,14 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                 const uint32_t trow = tmem + ((uint32_t)(q * 32) << 16) + b * kTcSlab + cq * 32;
                 mbar_wait(bar(kBarFReady + b), ph, ab, prm.status);
                 tc_fence_after();
-                float2 fr2[4];  // the weights of rows lane/4 + 8i of this warp's quarter, duplicated for the packed FMAs
-                {
-                    const float *f = fbuf + (b * 4 + cq) * kTcRows + q * 32 + (lane >> 2);
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) fr2[i] = make_float2(f[8 * i], f[8 * i]);
-                }
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {  // this warp's 32 columns of buffer half h
+                    float2 fr2[4];  // the weights of rows lane/4 + 8i for this chunk, duplicated for the packed FMAs
+                    {
+                        const float *f = fbuf + (b * 8 + h * 4 + cq) * kTcRows + q * 32 + (lane >> 2);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) fr2[i] = make_float2(f[8 * i], f[8 * i]);
+                    }
                     uint32_t va[16], vb[16];
                     tmem_ld_16x256b_x4(trow + h * 128, va);
                     tmem_ld_16x256b_x4(trow + h * 128 + (16u << 16), vb);
@@ -504,14 +492,17 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
             const int mt = item % prm.mtiles;
             const uint32_t b = k & 1, ph = (k >> 1) & 1;
             mbar_wait(bar(kBarEReady + b), ph, ab, prm.status);
-            // ---- merge the four column quarters of the row, publish the slab's statistics
-            float2 t4[4];
+            // ---- merge the eight chunks of the row, publish the slab's statistics
+            float cm[8];
+            float ms = -INFINITY;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) t4[i] = tstat[(b * 4 + i) * kTcRows + row];
-            const float ms = fmaxf(fmaxf(t4[0].x, t4[1].x), fmaxf(t4[2].x, t4[3].x));  // quarter 0 always holds a valid key
+            for (int i = 0; i < 8; ++i) {
+                cm[i] = tstat[(b * 8 + i) * kTcRows + row].x;
+                ms = fmaxf(ms, cm[i]);  // chunk 0 always holds a valid key
+            }
             float ls = 0.f;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) ls += (t4[i].x == -INFINITY) ? 0.f : t4[i].y * ex2(t4[i].x - ms);
+            for (int i = 0; i < 8; ++i) ls += (cm[i] == -INFINITY) ? 0.f : tstat[(b * 8 + i) * kTcRows + row].y * ex2(cm[i] - ms);
             st_gpu_f32x2(&prm.stats[((size_t)item * tasks_per_item + slab) * kTcRows + row], ms, ls * sgn);
 
             // ---- this row's statistics of every slab of the item; re-read until all carry this launch's mark
@@ -547,8 +538,8 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
             const bool row_valid = mt * kTcRows + row < prm.M;
             const float inv_l = row_valid ? 1.f / l : 0.f;
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
-                fbuf[(b * 4 + i) * kTcRows + row] = (t4[i].x == -INFINITY) ? 0.f : ex2(t4[i].x - m) * inv_l;
+            for (int i = 0; i < 8; ++i)
+                fbuf[(b * 8 + i) * kTcRows + row] = (cm[i] == -INFINITY) ? 0.f : ex2(cm[i] - m) * inv_l;
             mbar_arrive(bar(kBarFReady + b));
         }
     }
