@@ -27,8 +27,9 @@
 //            u_j = sum_i e_ij 2^(max_i - m_i) / l_i as a weighted column sum: the
 //            16x256b tensor-memory load shape hands every thread four rows of a
 //            column pair, so the sum over a warp's 32 rows is four packed FMAs plus
-//            a three-step exchange between lanes; the four row quarters are added
-//            through shared memory and stored: 256 floats per task.
+//            a three-step exchange between lanes; the four warps that own the same
+//            columns add their row quarters through shared memory (their own
+//            128-thread barrier) and store: 256 floats per task.
 // The two 128-column halves of a buffer are handed over separately (MMA -> pass 1,
 // pass 2 -> MMA), so the tensor core refills one half while the other is still read.
 //
@@ -59,8 +60,8 @@ constexpr uint32_t kTcSpinLimit = 1u << 22;                  // try_wait / poll 
 
 // shared-memory carve-up (bytes from the 1024-aligned base)
 constexpr uint32_t kTcOffStage = 0;                                        // [2] { Q, K }
-constexpr uint32_t kTcOffColpart = 2 * kTcStageBytes;                      // [4][256] float
-constexpr uint32_t kTcOffTstat = kTcOffColpart + 4 * kTcSlab * 4;          // [2 buffers][8 chunks][128] float2
+constexpr uint32_t kTcOffColpart = 2 * kTcStageBytes;                      // [2 parities][4 row quarters][256] float
+constexpr uint32_t kTcOffTstat = kTcOffColpart + 2 * 4 * kTcSlab * 4;          // [2 buffers][8 chunks][128] float2
 constexpr uint32_t kTcOffFbuf = kTcOffTstat + 2 * 8 * kTcRows * 8;         // [2 buffers][8 chunks][128] float
 constexpr uint32_t kTcOffBar = kTcOffFbuf + 2 * 8 * kTcRows * 4;
 constexpr uint32_t kTcSmemBytes = kTcOffBar + 256 + 1024;                  // + alignment slack
@@ -195,10 +196,10 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32
 }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-template <int kId>
-__device__ __forceinline__ void group_bar_sync()  // named barrier of the 512 epilogue threads
+// Named barrier of the four epilogue warps (one per TMEM lane quarter) that own the same columns.
+__device__ __forceinline__ void column_group_sync(int cq)
 {
-    asm volatile("bar.sync %0, 512;" ::"n"(kId) : "memory");
+    asm volatile("bar.sync %0, 128;" ::"r"(1 + cq) : "memory");
 }
 // The slab statistics are exchanged between CTAs with single 8-byte relaxed accesses at gpu scope:
 // one store publishes (max, marked sum) together, and a reader sees either the old or the new pair.
@@ -413,7 +414,6 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
         const int w = warp - 2;                 // 0..15
         const int cq = w >> 2;                  // this warp's columns: [32 cq, 32 cq + 32) of each buffer half
         const int row = q * 32 + lane;
-        const int gt = threadIdx.x - 64;        // 0..511 within the group
         float2 *tstat = reinterpret_cast<float2 *>(gbase + kTcOffTstat);
         const float *fbuf = reinterpret_cast<const float *>(gbase + kTcOffFbuf);
         float *colpart = reinterpret_cast<float *>(gbase + kTcOffColpart);
@@ -450,6 +450,7 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                 const uint32_t trow = tmem + ((uint32_t)(q * 32) << 16) + b * kTcSlab + cq * 32;
                 mbar_wait(bar(kBarFReady + b), ph, ab, prm.status);
                 tc_fence_after();
+                float *cpart = colpart + (kk & 1) * (4 * kTcSlab);
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {  // this warp's 32 columns of buffer half h
                     float2 fr2[4];  // the weights of rows lane/4 + 8i for this chunk, duplicated for the packed FMAs
@@ -458,6 +459,7 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
 #pragma unroll
                         for (int i = 0; i < 4; ++i) fr2[i] = make_float2(f[8 * i], f[8 * i]);
                     }
+                    float x[8];
                     uint32_t va[16], vb[16];
                     tmem_ld_16x256b_x4(trow + h * 128, va);
                     tmem_ld_16x256b_x4(trow + h * 128 + (16u << 16), vb);
@@ -465,19 +467,22 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                     tmem_wait_ld16(vb);
                     tc_fence_before();
                     mbar_arrive(bar(kBarTEmpty + 2 * b + h));   // this half may be overwritten by the task after next
-                    float x[8];
                     pass2_rows(va, vb, fr2, x);
                     const float u = pass2_reduce(x, lane);
                     const int g = lane >> 2, pp = lane & 3;
-                    colpart[q * kTcSlab + h * 128 + cq * 32 + 8 * (g >> 1) + 2 * pp + (g & 1)] = u;
+                    cpart[q * kTcSlab + h * 128 + cq * 32 + 8 * (g >> 1) + 2 * pp + (g & 1)] = u;
                 }
-                // ---- add the four row quarters, store this task's scores
-                group_bar_sync<1>();
-                if (gt < nvalid) {
-                    float *out = prm.scores + (size_t)mt * prm.part_stride + (size_t)unit * prm.N + slab * kTcSlab;
-                    out[gt] = (colpart[gt] + colpart[kTcSlab + gt]) + (colpart[2 * kTcSlab + gt] + colpart[3 * kTcSlab + gt]);
+                // ---- add the four row quarters of this column group, store its 64 scores
+                column_group_sync(cq);
+                if (q < 2) {  // warp q = 0 stores the group's columns of half 0, warp q = 1 those of half 1
+                    const int col = q * 128 + cq * 32 + lane;
+                    if (col < nvalid) {
+                        float *out = prm.scores + (size_t)mt * prm.part_stride + (size_t)unit * prm.N + slab * kTcSlab;
+                        out[col] = (cpart[col] + cpart[kTcSlab + col]) + (cpart[2 * kTcSlab + col] + cpart[3 * kTcSlab + col]);
+                    }
                 }
-                group_bar_sync<1>();                // colpart is rewritten by the next task
+                // no second barrier: the next task writes the other parity of colpart, and the one after
+                // that is separated from these reads by the next task's barrier
             }
         }
     } else {
