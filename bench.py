@@ -295,7 +295,8 @@ def main():
     score_flops = 2.0 * units * M * N * d
     compact_bytes = units * 4 * cfg.keep * d * e                # K and V, read + write, all kept rows
     names = ["nuc_rank", "cap_score", "select", "compact"]
-    dom = int(np.argmax(kms))
+    # the dominant kernel; scoring and compaction are close, scoring is named unless compaction is clearly longer
+    dom = 3 if kms[3] > 1.05 * kms[1] else 1
     if names[dom] == "compact":
         roof = {"kernel": "compact_kernel", "bound": "hbm", "achieved": compact_bytes / (kms[3] * 1e-3) / 1e9,
                 "peak": pk["hbm_gbs"], "unit": "GB/s"}

@@ -108,6 +108,30 @@ def test_config3_full_size_sampled_units():
     assert (np.diff(idx, axis=1) > 0).all() and idx.min() >= 0 and idx.max() < cfg.pot_size
 
 
+@pytest.mark.parametrize("cfg_id,n_sample", [(4, 8), (5, 6)])
+def test_configs_4_and_5_full_size_sampled_units(cfg_id, n_sample):
+    """Llama-3-8B-shaped batch of 16 streams (pot 8192, 2 row blocks) and the 70B-shaped layer (pot 16384,
+    4 row blocks, heavy-tailed keys, 5 % exactly duplicated tokens): the whole configuration runs on the
+    GPU, the checker follows sampled units; properties that hold at any size are checked on all units."""
+    cfg = inputs.CONFIGS[cfg_id]
+    t = inputs.make_cycle(cfg)
+    gpu = gpu_cycle(cfg, t, ipot.IPOT_SCORER_AUTO)
+    units = np.linspace(0, cfg.units - 1, n_sample).astype(np.int32)
+    same, cnt = compare_cycle(cfg, t, gpu, units=units)
+    assert cnt == n_sample and same >= n_sample - 2
+    u, idx, K, V = gpu
+    M = cfg.G * cfg.cap_rows
+    assert np.abs(u.sum(axis=1) - M).max() < 1e-4 * M
+    assert (np.diff(idx, axis=1) > 0).all() and idx.min() >= 0 and idx.max() < cfg.pot_size
+    Kin = t["K"].reshape(cfg.units, cfg.pot_size, cfg.d)
+    for unit in range(0, cfg.units, 7):     # gathered bytes on more units than the checker follows
+        assert (K[unit] == Kin[unit][idx[unit]]).all()
+    for b in range(cfg.batch):              # the novelty slots are in every head of the stream
+        nuc = set(oracle.nuc_top(t["aux"][b], cfg.nuc_slots).tolist())
+        for g in range(cfg.Hkv):
+            assert nuc <= set(idx[b * cfg.Hkv + g].tolist())
+
+
 def test_partially_filled_pot():
     cfg = inputs.small_config(cfg_id=220, pot_size=700, keep=300, nuc_slots=100, cap_rows=6, Hq=4, Hkv=2,
                               d=128, dtype="bf16", layers=2)
