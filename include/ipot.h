@@ -98,7 +98,9 @@ int ipot_set_nuc_slots(ipot_t *pot, int T);
 /* IPOT_SCORER_*; TENSOR is refused at the next cycle if the shape does not allow it. */
 int ipot_set_scorer(ipot_t *pot, int scorer);
 
-/* Forget the contents: len = 0.  Nothing is launched. */
+/* Forget the contents: len = 0.  Nothing is launched.  Also the way back to a defined state after
+ * ipot_sync_status() reported IPOT_E_TIMEOUT: the scorer's exchange buffers are cleared before their next use
+ * (the sticky status itself stays). */
 int ipot_reset(ipot_t *pot);
 
 /*

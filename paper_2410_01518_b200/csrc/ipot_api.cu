@@ -295,6 +295,7 @@ int ipot_reset(ipot_t *p)
 {
     if (!p) return IPOT_E_INVALID;
     p->len = 0;
+    p->tc.last_items = 0;  // the tensor scorer clears its statistics array before its next launch
     return IPOT_OK;
 }
 
