@@ -24,6 +24,7 @@ struct ipot {
     int sm_count;
     int scorer;
     int G, units, elem_bytes, row_bytes;
+    int compact_slices;
     cudaStream_t stream;
     // device memory (library-owned)
     void *K, *V;
@@ -95,8 +96,6 @@ int launch_simt(ipot *p, const void *Q, int M, int N)
 {
     const int d = p->cfg.d;
     const size_t smem = simt_smem_bytes(d);
-    IPOT_CUDA(cudaFuncSetAttribute(cap_row_stats<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)simt_smem_bytes(256)));
-    IPOT_CUDA(cudaFuncSetAttribute(cap_column_sums<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)simt_smem_bytes(256)));
     const float scale_log2e = (float)(1.4426950408889634 / std::sqrt((double)d));
     const size_t kstride = (size_t)p->cfg.pot_size * d;
     dim3 g1((M + kSimtRows - 1) / kSimtRows, p->units), g2((N + kSimtKeys - 1) / kSimtKeys, p->units);
@@ -120,7 +119,6 @@ int run_scoring(ipot *p, const void *Q, int cap_rows, const float *aux, int *par
     cudaEvent_t *ev = (p->profiling && p->ev_used < kProfSlots) ? p->ev[p->ev_used] : nullptr;
     if (ev) IPOT_CUDA(cudaEventRecord(ev[0], p->stream));
     if (T > 0 && aux) {
-        IPOT_CUDA(cudaFuncSetAttribute(nuc_mask_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 32768 * 4));
         nuc_mask_kernel<<<p->cfg.batch, kSelThreads, (size_t)N * 4, p->stream>>>(aux, p->nuc_mask, N, T);
         p->launches += 1;
         IPOT_CUDA(cudaGetLastError());
@@ -153,12 +151,10 @@ int check_cycle_args(ipot *p, const void *Q, int cap_rows, const float *aux, boo
     return IPOT_OK;
 }
 
+// Byte-column slices per row for the compaction grid: enough blocks to fill the device, slices of >= 64 bytes.
 int compact_slices(const ipot *p)
 {
     const int row_vecs = p->row_bytes / 16;
-    const char *env = getenv("IPOT_COMPACT_SLICES");
-    const int want = env ? atoi(env) : 0;
-    if (want > 0 && row_vecs % want == 0) return want;
     int slices = 1;
     while (row_vecs % (slices * 2) == 0 && row_vecs / (slices * 2) >= 4 &&
            (long long)p->units * 2 * slices < 8LL * p->sm_count)
@@ -174,7 +170,6 @@ int run_cycle(ipot *p, const void *Q, int cap_rows, const float *aux)
     int rc = run_scoring(p, Q, cap_rows, aux, &parts);
     if (rc != IPOT_OK) return rc;
     const size_t part_stride = (size_t)p->units * p->cfg.pot_size;
-    IPOT_CUDA(cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 32768 * 4));
     select_kernel<<<p->units, kSelThreads, (size_t)N * 4, p->stream>>>(
         p->scores, parts, part_stride, T > 0 ? p->nuc_mask : nullptr, p->idx,
         parts > 1 ? p->summed : nullptr, N, keep, p->cfg.Hkv, p->cfg.batch, p->status);
@@ -183,7 +178,7 @@ int run_cycle(ipot *p, const void *Q, int cap_rows, const float *aux)
     if (ev) IPOT_CUDA(cudaEventRecord(ev[3], p->stream));
 
     const int row_vecs = p->row_bytes / 16;
-    const int slices = compact_slices(p);
+    const int slices = p->compact_slices;
     dim3 grid(slices, p->units, 2);
     compact_kernel<<<grid, kMoveThreads, 0, p->stream>>>((uint4 *)p->K, (uint4 *)p->V, p->idx, keep, N, row_vecs,
                                                         row_vecs / slices, (size_t)p->cfg.pot_size * row_vecs, p->status);
@@ -256,6 +251,20 @@ int ipot_create_ex(const ipot_config_t *cfg, ipot_t **out)
         delete p;
         return IPOT_E_NOMEM;
     }
+    // kernels whose dynamic shared memory can exceed the default limit
+    ok = cudaFuncSetAttribute(cap_row_stats<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)simt_smem_bytes(256)) == cudaSuccess &&
+         cudaFuncSetAttribute(cap_column_sums<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)simt_smem_bytes(256)) == cudaSuccess &&
+         cudaFuncSetAttribute(cap_row_stats<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)simt_smem_bytes(256)) == cudaSuccess &&
+         cudaFuncSetAttribute(cap_column_sums<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)simt_smem_bytes(256)) == cudaSuccess &&
+         cudaFuncSetAttribute(nuc_mask_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 32768 * 4) == cudaSuccess &&
+         cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 32768 * 4) == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        free_all(p);
+        delete p;
+        return IPOT_E_CUDA;
+    }
+    p->compact_slices = compact_slices(p);
     tc_plan_init(p->tc, p->cfg, p->K, p->sm_count);
     *out = p;
     return IPOT_OK;
