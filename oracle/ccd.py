@@ -30,10 +30,13 @@ def _load():
         lib.ora_gather.argtypes = [bp, C.c_size_t, ip, C.c_int, bp]
         lib.ora_cycle.argtypes = [dp, dp, bp, bp, dp, ip, C.c_int, C.c_int, C.c_int, C.c_int,
                                   C.c_int, C.c_int, C.c_int, C.c_size_t, dp, ip, bp, bp]
+        lib.ora_cap_scores_incl.argtypes = [dp, dp, dp, C.c_int, C.c_int, C.c_int, C.c_int, dp, dp]
+        lib.ora_cycle_cap.argtypes = [dp, dp, dp, bp, bp, dp, ip, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
+                                      C.c_int, C.c_int, C.c_int, C.c_size_t, dp, ip, bp, bp]
         lib.ora_set_threads.argtypes = [C.c_int]
         lib.ora_max_threads.restype = C.c_int
         for f in (lib.ora_nuc_top, lib.ora_cap_scores, lib.ora_select, lib.ora_gather,
-                  lib.ora_cycle, lib.ora_set_threads):
+                  lib.ora_cycle, lib.ora_set_threads, lib.ora_cap_scores_incl, lib.ora_cycle_cap):
             f.restype = None
         _lib = lib
     return _lib
@@ -86,6 +89,20 @@ def cap_scores(Q, K, return_row_sums: bool = False):
     return (u, rs) if return_row_sums else u
 
 
+def cap_scores_incl(Q, K, Kc, P: int, return_pot_mass: bool = False):
+    """Appendix B listing read literally, one KV head: Q [G*P][d], K [N][d], Kc [P][d] (float64) -> u [N].
+    Row r sees the pot keys and the CaP keys 0..r % P; only the pot columns are summed."""
+    Q, K, Kc = _f64(Q), _f64(K), _f64(Kc)
+    M, d = Q.shape
+    N = K.shape[0]
+    assert K.shape[1] == d and Kc.shape == (P, d) and M % P == 0
+    u = np.empty(N, dtype=np.float64)
+    pm = np.empty(M, dtype=np.float64)
+    _load().ora_cap_scores_incl(_p(Q, C.c_double), _p(K, C.c_double), _p(Kc, C.c_double), M, N, d, P,
+                                _p(u, C.c_double), _p(pm, C.c_double))
+    return (u, pm) if return_pot_mass else u
+
+
 def select(u, nuc, keep: int) -> np.ndarray:
     """Sec. 3.3.3 / Appendix B: NuC slots + best (keep - T) other slots, ascending."""
     u = _f64(u)
@@ -107,13 +124,14 @@ def gather(rows: np.ndarray, idx) -> np.ndarray:
     return out
 
 
-def cycle(Q, K, V, aux, keep: int, T: int, units=None, with_kv: bool = True):
+def cycle(Q, K, V, aux, keep: int, T: int, units=None, with_kv: bool = True, K_cap=None):
     """One CCD cycle over all (or the listed) units.
 
     Q [L][B][Hq][P][d], K, V [L][B][Hkv][N][d] in storage dtype (float32 or
     uint16 bfloat16 bits), aux [B][N].  ``units`` lists flat unit indices
     ``(l*B + b)*Hkv + g``.  Returns a dict with ``units``, ``u`` [n][N],
     ``idx`` [n][keep] and, if ``with_kv``, the compacted ``K``, ``V`` [n][keep][d].
+    With ``K_cap`` [L][B][Hkv][P][d] the scores are the CaP-inclusive ones.
     """
     L, B, Hq, P, d = Q.shape
     Hkv, N = K.shape[2], K.shape[3]
@@ -131,6 +149,10 @@ def cycle(Q, K, V, aux, keep: int, T: int, units=None, with_kv: bool = True):
     Vs = np.ascontiguousarray(Vf[units])
     Qd = widen_storage(Qf[units])
     Kd = widen_storage(Ks)
+    Kcd = None
+    if K_cap is not None:
+        assert K_cap.shape == (L, B, Hkv, P, d)
+        Kcd = widen_storage(np.ascontiguousarray(K_cap).reshape(all_units, P, d)[units])
     auxd = _f64(aux)
     assert auxd.shape == (B, N)
     stream_of = np.ascontiguousarray((units // Hkv) % B, dtype=np.int32)
@@ -140,9 +162,9 @@ def cycle(Q, K, V, aux, keep: int, T: int, units=None, with_kv: bool = True):
     Ko = np.empty((n, keep, d), dtype=Ks.dtype) if with_kv else None
     Vo = np.empty((n, keep, d), dtype=Vs.dtype) if with_kv else None
     bp = C.POINTER(C.c_uint8)
-    _load().ora_cycle(
-        _p(Qd, C.c_double), _p(Kd, C.c_double),
+    _load().ora_cycle_cap(
+        _p(Qd, C.c_double), _p(Kd, C.c_double), _p(Kcd, C.c_double) if Kcd is not None else None,
         Ks.ctypes.data_as(bp), Vs.ctypes.data_as(bp), _p(auxd, C.c_double), _p(stream_of, C.c_int),
-        n, B, M, d, N, keep, T, rb, _p(u, C.c_double), _p(idx, C.c_int),
+        n, B, M, P, d, N, keep, T, rb, _p(u, C.c_double), _p(idx, C.c_int),
         Ko.ctypes.data_as(bp) if with_kv else None, Vo.ctypes.data_as(bp) if with_kv else None)
     return {"units": units, "u": u, "idx": idx, "K": Ko, "V": Vo}

@@ -15,7 +15,12 @@
  *                    slots by CaP score, per head
  *   ora_gather       Appendix B "KV-cache compression": K and V rows of the
  *                    retained slots
+ *   ora_cap_scores_incl  the variant the Appendix B listing spells out: the CaP
+ *                    queries attend to the pot keys AND, causally, to the CaP's
+ *                    own keys; the CaP columns are then cut away, so they only
+ *                    take probability mass from the pot columns
  *   ora_cycle        the four steps over every (layer, stream, kv-head) unit
+ *   ora_cycle_cap    the same with the CaP-inclusive scores
  *
  * Readings where the paper is silent (each listed in the design notes):
  *   - every CaP row normalises over the N pot keys only (CaP keys are not in
@@ -28,11 +33,16 @@
  *   - ties: the lower slot index wins, in both rankings;
  *   - survivors keep their original order (ascending slot index).
  *
+ *   - CaP-inclusive variant: CaP row i (0-based, within its query head) sees the
+ *     CaP keys 0..i of its KV head (causal mask), all of them after every pot key;
  * Parity pins (tests/test_oracle_pins.py): row sums = 1, column-sum total =
  * G*P, closed forms (Q = 0, equal keys, N = 1, one dominant key), slot
  * permutation equivariance, P=G=1 against an independent library softmax,
  * brute-force subset enumeration for the selection on tiny pots, NuC-only and
- * CaP-only special cases, byte-wise gather identities.
+ * CaP-only special cases, byte-wise gather identities.  CaP-inclusive variant:
+ * Q = 0 closed form G * sum_i 1/(N+i+1), masked library softmax over the N+P
+ * columns, far-away CaP keys reduce it to ora_cap_scores, a later CaP key never
+ * changes an earlier row.
  */
 #include <math.h>
 #include <stdint.h>
@@ -99,6 +109,40 @@ void ora_cap_scores(const double *Q, const double *K, int M, int N, int d,
 }
 
 /*
+ * Appendix B "Calculate Attention Score", read literally.  Row r of Q belongs to CaP
+ * position i = r % P of one of the G query heads; Kc holds the P CaP keys of the KV
+ * head ([P][d]).  The row's softmax runs over the N pot keys and the CaP keys 0..i;
+ * only the pot columns are added into u.  pot_mass (may be NULL) receives, per row,
+ * the probability that stayed on the pot columns (1 minus what the CaP keys took).
+ */
+void ora_cap_scores_incl(const double *Q, const double *K, const double *Kc, int M, int N, int d,
+                         int P, double *u, double *pot_mass)
+{
+    double *s = (double *)malloc(sizeof(double) * (size_t)(N + P));
+    const double scale = 1.0 / sqrt((double)d);
+    for (int j = 0; j < N; ++j) u[j] = 0.0;
+    for (int r = 0; r < M; ++r) {
+        const double *q = Q + (size_t)r * d;
+        const int i = r % P;          /* CaP position of this row */
+        const int n = N + i + 1;      /* columns this row may see */
+        double m = -INFINITY;
+        for (int j = 0; j < n; ++j) {
+            const double *k = (j < N) ? K + (size_t)j * d : Kc + (size_t)(j - N) * d;
+            double acc = 0.0;
+            for (int c = 0; c < d; ++c) acc += q[c] * k[c];
+            s[j] = acc * scale;
+            if (s[j] > m) m = s[j];
+        }
+        double Z = 0.0;
+        for (int j = 0; j < n; ++j) { s[j] = exp(s[j] - m); Z += s[j]; }
+        double pm = 0.0;
+        for (int j = 0; j < N; ++j) { double p = s[j] / Z; u[j] += p; pm += p; }
+        if (pot_mass) pot_mass[r] = pm;
+    }
+    free(s);
+}
+
+/*
  * Per-head selection.  nuc[0..T) are the NuC slots of the stream (they are kept
  * in every head); of the other slots the R = keep - T with the largest u are
  * kept (ties: lower slot first).  idx[0..keep) is returned ascending.
@@ -139,10 +183,11 @@ void ora_gather(const uint8_t *rows, size_t row_bytes, const int *idx, int keep,
  *   Kout, Vout [n_units][keep][row_bytes]  (may be NULL)
  * Units are independent; with OpenMP one thread takes one unit at a time.
  */
-void ora_cycle(const double *Qd, const double *Kd, const uint8_t *Kb, const uint8_t *Vb,
-               const double *aux, const int *stream_of, int n_units, int B, int M, int d,
-               int N, int keep, int T, size_t row_bytes,
-               double *u_out, int *idx_out, uint8_t *Kout, uint8_t *Vout)
+/* Kcd: [n_units][P][d] double CaP keys, or NULL for the context-only softmax of ora_cycle. */
+void ora_cycle_cap(const double *Qd, const double *Kd, const double *Kcd, const uint8_t *Kb,
+                   const uint8_t *Vb, const double *aux, const int *stream_of, int n_units, int B,
+                   int M, int P, int d, int N, int keep, int T, size_t row_bytes,
+                   double *u_out, int *idx_out, uint8_t *Kout, uint8_t *Vout)
 {
     int *nuc = (int *)malloc(sizeof(int) * (size_t)B * (size_t)(T > 0 ? T : 1));
     for (int b = 0; b < B; ++b) ora_nuc_top(aux + (size_t)b * N, N, T, nuc + (size_t)b * T);
@@ -152,7 +197,8 @@ void ora_cycle(const double *Qd, const double *Kd, const uint8_t *Kb, const uint
         const double *K = Kd + (size_t)t * N * d;
         double *u = u_out + (size_t)t * N;
         int *idx = idx_out + (size_t)t * keep;
-        ora_cap_scores(Q, K, M, N, d, u, NULL);
+        if (Kcd) ora_cap_scores_incl(Q, K, Kcd + (size_t)t * P * d, M, N, d, P, u, NULL);
+        else ora_cap_scores(Q, K, M, N, d, u, NULL);
         ora_select(u, N, nuc + (size_t)stream_of[t] * T, T, keep, idx);
         if (Kout) ora_gather(Kb + (size_t)t * N * row_bytes, row_bytes, idx, keep,
                              Kout + (size_t)t * keep * row_bytes);
@@ -160,6 +206,15 @@ void ora_cycle(const double *Qd, const double *Kd, const uint8_t *Kb, const uint
                              Vout + (size_t)t * keep * row_bytes);
     }
     free(nuc);
+}
+
+void ora_cycle(const double *Qd, const double *Kd, const uint8_t *Kb, const uint8_t *Vb,
+               const double *aux, const int *stream_of, int n_units, int B, int M, int d,
+               int N, int keep, int T, size_t row_bytes,
+               double *u_out, int *idx_out, uint8_t *Kout, uint8_t *Vout)
+{
+    ora_cycle_cap(Qd, Kd, NULL, Kb, Vb, aux, stream_of, n_units, B, M, 1, d, N, keep, T, row_bytes,
+                  u_out, idx_out, Kout, Vout);
 }
 
 /* Thread count used by ora_cycle (1 when built without OpenMP). */

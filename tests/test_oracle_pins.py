@@ -251,3 +251,81 @@ def test_cycle_accepts_bf16_bit_patterns():
     bits = torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
     wide = oracle.widen_storage(bits)
     assert (wide == torch.from_numpy(x).to(torch.bfloat16).to(torch.float64).numpy()).all()
+
+
+# ---------------------------------------------------------------- Appendix B listing, CaP keys inside the softmax
+def test_incl_zero_queries_closed_form():
+    # all logits 0: CaP position i sees N + i + 1 columns, each pot column gets 1 / (N + i + 1)
+    g = rnd(50)
+    G, P, N, d = 3, 4, 7, 8
+    u, pm = oracle.cap_scores_incl(np.zeros((G * P, d)), g.standard_normal((N, d)), g.standard_normal((P, d)), P, True)
+    want = G * sum(Fraction(1, N + i + 1) for i in range(P))
+    np.testing.assert_allclose(u, float(want), rtol=1e-14)
+    np.testing.assert_allclose(pm, [N / (N + (r % P) + 1) for r in range(G * P)], rtol=1e-14)
+
+
+def test_incl_against_masked_library_softmax():
+    torch = pytest.importorskip("torch")
+    g = rnd(51)
+    G, P, N, d = 2, 5, 40, 16
+    Q, K, Kc = g.standard_normal((G * P, d)) * 2, g.standard_normal((N, d)) * 2, g.standard_normal((P, d)) * 2
+    logits = torch.from_numpy(np.concatenate([Q @ K.T, Q @ Kc.T], axis=1) / np.sqrt(d))
+    pos = torch.arange(G * P) % P                                # CaP position of each row
+    hidden = torch.arange(P)[None, :] > pos[:, None]             # CaP key i' is hidden from row i when i' > i
+    logits[:, N:] = logits[:, N:].masked_fill(hidden, float("-inf"))
+    p = torch.softmax(logits, dim=1).numpy()
+    u, pm = oracle.cap_scores_incl(Q, K, Kc, P, True)
+    np.testing.assert_allclose(u, p[:, :N].sum(axis=0), rtol=1e-12)
+    np.testing.assert_allclose(pm, p[:, :N].sum(axis=1), rtol=1e-12)
+    assert abs(u.sum() + p[:, N:].sum() - G * P) < 1e-10         # the CaP columns took the rest
+
+
+def test_incl_far_away_cap_keys_reduce_to_eq2():
+    g = rnd(52)
+    G, P, N, d = 2, 3, 25, 8
+    Q = np.abs(g.standard_normal((G * P, d))) + 0.1               # every q . (-c 1) is very negative
+    K = g.standard_normal((N, d))
+    Kc = -400.0 * np.ones((P, d))
+    np.testing.assert_allclose(oracle.cap_scores_incl(Q, K, Kc, P), oracle.cap_scores(Q, K), rtol=1e-12)
+
+
+def test_incl_is_causal_inside_the_cap():
+    g = rnd(53)
+    G, P, N, d = 2, 4, 12, 8
+    Q, K, Kc = g.standard_normal((G * P, d)), g.standard_normal((N, d)), g.standard_normal((P, d))
+    _, pm = oracle.cap_scores_incl(Q, K, Kc, P, True)
+    Kc2 = Kc.copy()
+    Kc2[2] += 3.0                                                 # only rows at CaP positions 2 and 3 may notice
+    _, pm2 = oracle.cap_scores_incl(Q, K, Kc2, P, True)
+    for r in range(G * P):
+        assert (pm[r] == pm2[r]) == (r % P < 2)
+    # a single CaP row (P = 1) sees exactly one CaP key: its own
+    q, kc = Q[:1], Kc[:1]
+    s = np.concatenate([K @ q[0], kc @ q[0]]) / np.sqrt(d)
+    e = np.exp(s - s.max())
+    np.testing.assert_allclose(oracle.cap_scores_incl(q, K, kc, 1), (e / e.sum())[:N], rtol=1e-12)
+
+
+def test_cycle_with_cap_keys_wiring():
+    g = rnd(54)
+    L, B, Hq, Hkv, P, d, N, keep, T = 2, 2, 4, 2, 3, 8, 20, 9, 4
+    G = Hq // Hkv
+    Q = g.standard_normal((L, B, Hq, P, d)).astype(np.float32)
+    K = g.standard_normal((L, B, Hkv, N, d)).astype(np.float32)
+    V = g.standard_normal((L, B, Hkv, N, d)).astype(np.float32)
+    Kc = g.standard_normal((L, B, Hkv, P, d)).astype(np.float32)
+    aux = g.random((B, N)).astype(np.float32)
+    out = oracle.cycle(Q, K, V, aux, keep, T, K_cap=Kc)
+    for l in range(L):
+        for b in range(B):
+            for kv in range(Hkv):
+                unit = (l * B + b) * Hkv + kv
+                u = sum(oracle.cap_scores_incl(Q[l, b, h].astype(np.float64), K[l, b, kv].astype(np.float64),
+                                               Kc[l, b, kv].astype(np.float64), P)
+                        for h in range(Hq) if h // G == kv)
+                np.testing.assert_allclose(out["u"][unit], u, rtol=1e-12)
+                assert out["u"][unit].sum() < G * P
+                assert (out["idx"][unit] == oracle.select(out["u"][unit], oracle.nuc_top(aux[b], T), keep)).all()
+                assert (out["K"][unit] == K[l, b, kv][out["idx"][unit]]).all()
+    base = oracle.cycle(Q, K, V, aux, keep, T)
+    assert not np.allclose(base["u"], out["u"])
