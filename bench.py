@@ -48,12 +48,15 @@ def workload_shape(cfg):
     return n_new, cfg.pot_size
 
 
-def gen_ring(cfg, n_new):
-    """RING chunks of new K/V rows, CaP queries and novelty scores (numpy, storage dtype)."""
+def gen_ring(cfg, n_new, cap_keys=False):
+    """RING chunks of new K/V rows, CaP queries and novelty scores (numpy, storage dtype);
+    with cap_keys also the CaP's own key rows (CaP-inclusive scoring)."""
     ring = []
     for i in range(RING):
         K, V = inputs.make_kv(cfg, n_new, chunk=1 + i)
         ring.append({"K": K, "V": V, "Q": inputs.make_q(cfg, 1 + i), "aux": inputs.make_aux(cfg, 1 + i)})
+        if cap_keys:
+            ring[-1]["K_cap"] = inputs.make_kcap(cfg, 1 + i)
     K0, V0 = inputs.make_kv(cfg, cfg.keep, chunk=0)
     return ring, K0, V0
 
@@ -116,9 +119,9 @@ def cpu_baseline(cfg, ring, K0, V0, n_units_sample, threads=None):
     K = np.concatenate([K0, t["K"]], axis=3)
     V = np.concatenate([V0, t["V"]], axis=3)
     units = np.linspace(0, cfg.units - 1, n_units_sample).astype(np.int32)
-    oracle.cycle(t["Q"], K, V, t["aux"], cfg.keep, cfg.nuc_slots, units=units[:1])  # load the library
+    oracle.cycle(t["Q"], K, V, t["aux"], cfg.keep, cfg.nuc_slots, units=units[:1], K_cap=t.get("K_cap"))  # load the library
     t0 = time.perf_counter()
-    oracle.cycle(t["Q"], K, V, t["aux"], cfg.keep, cfg.nuc_slots, units=units)
+    oracle.cycle(t["Q"], K, V, t["aux"], cfg.keep, cfg.nuc_slots, units=units, K_cap=t.get("K_cap"))
     dt = time.perf_counter() - t0
     cycles_per_s = (len(units) / cfg.units) / dt
     return cycles_per_s, dt, len(units), oracle.max_threads()
@@ -143,7 +146,7 @@ def run_reference(args, cfg):
         return
     n_new, N = workload_shape(cfg)
     small = cfg.with_layers(min(cfg.layers, 2))  # the sample only needs a few layers' tensors
-    ring, K0, V0 = gen_ring(small, n_new)
+    ring, K0, V0 = gen_ring(small, n_new, args.cap_keys)
     n_sample = min(small.units, 16)
     for _ in range(args.warmup):
         cpu_baseline(small, ring, K0, V0, 1)
@@ -157,7 +160,7 @@ def run_reference(args, cfg):
         "impl": "reference", "metric": "ccd_cycles_per_s", "value": value, "unit": "cycles/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": config_dict(cfg, n_new, N),
+        "config": config_dict(cfg, n_new, N, args.cap_keys),
         "cpu_baseline": {"value": value, "unit": "cycles/s", "cores": threads, "kind": "oracle",
                          "sample": f"{n_sample} of {cfg.units} units of one cycle per step (units are independent and "
                                    f"equal-sized); full-cycle time extrapolated"},
@@ -167,9 +170,10 @@ def run_reference(args, cfg):
     print(json.dumps(line))
 
 
-def config_dict(cfg, n_new, N):
+def config_dict(cfg, n_new, N, cap_keys=False):
     return {"workload": f"configs[{cfg.cfg_id - 1}] {cfg.name}: one CCD cycle per step "
-                        f"(append {n_new} rows, distil {N} -> {cfg.keep})",
+                        f"(append {n_new} rows, distil {N} -> {cfg.keep})"
+                        + ("; CaP keys inside the softmax" if cap_keys else ""),
             "layers": cfg.layers, "batch": cfg.batch, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "d": cfg.d,
             "pot_size": cfg.pot_size, "keep": cfg.keep, "nuc_slots": cfg.nuc_slots, "cap_rows": cfg.cap_rows,
             "units": cfg.units, "l2": "inputs_larger_than_l2" if cfg.units * N * cfg.d * cfg.elem_bytes * 2 > 126e6
@@ -185,6 +189,8 @@ def main():
     ap.add_argument("--workload", default="cfg3", choices=sorted(WORKLOADS))
     ap.add_argument("--scorer", default="auto", choices=["auto", "simt", "tensor"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cap-keys", action="store_true",
+                    help="score with the CaP's own keys inside the softmax (the Appendix B listing read literally)")
     ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (profiling small cases)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -209,7 +215,7 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     n_new, N = workload_shape(cfg)
-    ring, K0, V0 = gen_ring(cfg, n_new)
+    ring, K0, V0 = gen_ring(cfg, n_new, args.cap_keys)
     tdt = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
 
     def dev(a):
@@ -240,12 +246,18 @@ def main():
         if flush is not None:
             flush.add_(1)
         ipot.ipot_append_chunk(h, t["K"], t["V"], n_new)
-        ipot.ipot_score_and_compress(h, t["Q"], cfg.cap_rows, t["aux"])
+        if args.cap_keys:
+            ipot.ipot_score_and_compress_cap(h, t["Q"], t["K_cap"], cfg.cap_rows, t["aux"])
+        else:
+            ipot.ipot_score_and_compress(h, t["Q"], cfg.cap_rows, t["aux"])
 
     def step_host(i):
         t = hring[i % RING]
         ipot.ipot_append_chunk_host(h, t["K"], t["V"], n_new)
-        ipot.ipot_score_and_compress_host(h, t["Q"], cfg.cap_rows, t["aux"], idx_host)
+        if args.cap_keys:
+            ipot.ipot_score_and_compress_cap_host(h, t["Q"], t["K_cap"], cfg.cap_rows, t["aux"], idx_host)
+        else:
+            ipot.ipot_score_and_compress_host(h, t["Q"], cfg.cap_rows, t["aux"], idx_host)
 
     def barrier():
         if world > 1:
@@ -285,7 +297,7 @@ def main():
     e2e_steps = max(3, min(args.steps, 50))
     e2e_value, _, _, _ = timed(step_host, e2e_steps, 3)
     assert ipot.ipot_sync_status(h) == 0
-    h2d = sum(hring[0][k].numel() * hring[0][k].element_size() for k in ("K", "V", "Q", "aux"))
+    h2d = sum(v.numel() * v.element_size() for v in hring[0].values())
     d2h = idx_host.numel() * 4
 
     # roofline of the dominant kernel
@@ -318,7 +330,7 @@ def main():
         "metric": "ccd_cycles_per_s", "value": value, "unit": "cycles/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
-        "config": config_dict(cfg, n_new, N),
+        "config": config_dict(cfg, n_new, N, args.cap_keys),
         "pot_tokens_per_s": value * N * cfg.batch,
         "layer_cycles_per_s": value * cfg.layers,
         "clocks": clocks,

@@ -148,6 +148,29 @@ int ipot_score_and_compress_host(ipot_t *pot, const void *Q_cap_host, int cap_ro
 int ipot_score_only(ipot_t *pot, const void *Q_cap, int cap_rows, const float *aux_scores);
 
 /*
+ * The cycle with the CaP's own keys inside the softmax, as the PyTorch-style
+ * listing of Appendix B ("Calculate Attention Score") computes it: the CaP
+ * queries attend to every key of the sequence, the CaP included, under the
+ * causal mask, and the CaP columns are cut away before the rows are summed.
+ * CaP row i (0-based, within its query head) therefore normalises over the len
+ * pot keys and the CaP keys 0..i of its KV head; the scores of a unit then sum to
+ * less than G * cap_rows.  Selection and compaction are unchanged.
+ *   K_cap : device, [layers][batch][Hkv][cap_rows][d], pot dtype, 16-byte
+ *           aligned, caller-owned, read-only; the keys of the same cap_rows
+ *           positions the queries of Q_cap belong to.
+ * Everything else as in ipot_score_and_compress / ipot_score_only; a NULL K_cap
+ * is IPOT_E_INVALID (use the plain calls for the context-only softmax).
+ */
+int ipot_score_and_compress_cap(ipot_t *pot, const void *Q_cap, const void *K_cap, int cap_rows,
+                                const float *aux_scores);
+int ipot_score_only_cap(ipot_t *pot, const void *Q_cap, const void *K_cap, int cap_rows,
+                        const float *aux_scores);
+/* ipot_score_and_compress_cap with HOST buffers (Q_cap, K_cap, aux staged on the device first; index
+ * lists copied back if idx_host is not NULL), as ipot_score_and_compress_host. */
+int ipot_score_and_compress_cap_host(ipot_t *pot, const void *Q_cap_host, const void *K_cap_host, int cap_rows,
+                                     const float *aux_host, int32_t *idx_host);
+
+/*
  * Borrowed device pointers to the pot ([layers][batch][Hkv][pot_size][d]) and
  * the current fill.  Rows >= len are undefined.  The pointers stay valid until
  * ipot_destroy(); their contents are final once the stream's queued work ran.

@@ -10,6 +10,7 @@
 #include <new>
 
 #include "common.cuh"
+#include "k_cap_self.cuh"
 #include "k_move.cuh"
 #include "k_score_simt.cuh"
 #include "k_score_tc.cuh"
@@ -33,10 +34,12 @@ struct ipot {
     float *summed;       // [units][N]: sum of the partial arrays when there are several
     int max_parts;
     float2 *row_stats;   // [units][max M]
+    float2 *cap_stats;   // [units][max M]: (max, sum) over the CaP's own keys, CaP-inclusive scoring only
     uint8_t *nuc_mask;   // [batch][pot_size]
     int32_t *idx;        // [units][keep]
     int *status;         // sticky device status word
     void *stage_q;       // device staging for the *_host calls
+    void *stage_kc;
     float *stage_aux;
     // results of the last cycle
     int last_len_before;
@@ -82,8 +85,8 @@ void free_all(ipot *p)
 {
     tc_plan_destroy(p->tc);
     cudaFree(p->K); cudaFree(p->V); cudaFree(p->scores); cudaFree(p->summed);
-    cudaFree(p->row_stats); cudaFree(p->nuc_mask); cudaFree(p->idx); cudaFree(p->status);
-    cudaFree(p->stage_q); cudaFree(p->stage_aux);
+    cudaFree(p->row_stats); cudaFree(p->cap_stats); cudaFree(p->nuc_mask); cudaFree(p->idx); cudaFree(p->status);
+    cudaFree(p->stage_q); cudaFree(p->stage_kc); cudaFree(p->stage_aux);
     if (p->ev) {
         for (int i = 0; i < kProfSlots; ++i)
             for (auto &e : p->ev[i]) if (e) cudaEventDestroy(e);
@@ -91,15 +94,39 @@ void free_all(ipot *p)
     }
 }
 
+// Row statistics over the CaP's own keys (causal): what Appendix B's listing adds to every row's denominator.
+int launch_cap_self(ipot *p, const void *Q, const void *Kc, int M, int P)
+{
+    const int d = p->cfg.d;
+    const float scale_log2e = (float)(1.4426950408889634 / std::sqrt((double)d));
+    if (p->cfg.dtype == IPOT_BF16 && d % 16 == 0) {
+        dim3 g((M + kSelfRows - 1) / kSelfRows, p->units);
+        cap_self_stats_bf16<<<g, kSelfWarps * 32, self_smem_bytes(d), p->stream>>>((const __nv_bfloat16 *)Q, (const __nv_bfloat16 *)Kc, p->cap_stats,
+                                                                 M, P, d, scale_log2e);
+    } else {
+        dim3 g((M + kSimtRows - 1) / kSimtRows, p->units);
+        if (p->cfg.dtype == IPOT_F32)
+            cap_row_stats<float><<<g, kSimtThreads, simt_smem_bytes(d), p->stream>>>(
+                (const float *)Q, (const float *)Kc, p->cap_stats, M, P, d, (size_t)P * d, scale_log2e, nullptr, P, 0);
+        else
+            cap_row_stats<__nv_bfloat16><<<g, kSimtThreads, simt_smem_bytes(d), p->stream>>>(
+                (const __nv_bfloat16 *)Q, (const __nv_bfloat16 *)Kc, p->cap_stats, M, P, d, (size_t)P * d, scale_log2e, nullptr, P, 0);
+    }
+    p->launches += 1;
+    IPOT_CUDA(cudaGetLastError());
+    return IPOT_OK;
+}
+
 template <typename T>
-int launch_simt(ipot *p, const void *Q, int M, int N)
+int launch_simt(ipot *p, const void *Q, const float2 *cap_stats, int M, int N)
 {
     const int d = p->cfg.d;
     const size_t smem = simt_smem_bytes(d);
     const float scale_log2e = (float)(1.4426950408889634 / std::sqrt((double)d));
     const size_t kstride = (size_t)p->cfg.pot_size * d;
     dim3 g1((M + kSimtRows - 1) / kSimtRows, p->units), g2((N + kSimtKeys - 1) / kSimtKeys, p->units);
-    cap_row_stats<T><<<g1, kSimtThreads, smem, p->stream>>>((const T *)Q, (const T *)p->K, p->row_stats, M, N, d, kstride, scale_log2e);
+    cap_row_stats<T><<<g1, kSimtThreads, smem, p->stream>>>((const T *)Q, (const T *)p->K, p->row_stats, M, N, d, kstride, scale_log2e,
+                                                            cap_stats, 0, 1);
     cap_column_sums<T><<<g2, kSimtThreads, smem, p->stream>>>((const T *)Q, (const T *)p->K, p->row_stats, p->scores, M, N, d, kstride, scale_log2e);
     p->launches += 2;
     IPOT_CUDA(cudaGetLastError());
@@ -108,7 +135,7 @@ int launch_simt(ipot *p, const void *Q, int M, int N)
 
 // Steps 1-2 (and the timing events around them).  On success *parts tells how many
 // partial score arrays the scorer wrote.
-int run_scoring(ipot *p, const void *Q, int cap_rows, const float *aux, int *parts)
+int run_scoring(ipot *p, const void *Q, const void *Kc, int cap_rows, const float *aux, int *parts)
 {
     const int N = p->len, T = p->cfg.nuc_slots, M = p->G * cap_rows;
     int scorer = p->scorer;
@@ -126,13 +153,18 @@ int run_scoring(ipot *p, const void *Q, int cap_rows, const float *aux, int *par
     if (ev) IPOT_CUDA(cudaEventRecord(ev[1], p->stream));
     *parts = 1;
     int rc;
+    if (Kc) {
+        rc = launch_cap_self(p, Q, Kc, M, cap_rows);
+        if (rc != IPOT_OK) return rc;
+    }
+    const float2 *cap_stats = Kc ? p->cap_stats : nullptr;
     if (scorer == IPOT_SCORER_TENSOR) {
         int n_launch = 0;
-        rc = tc_launch(p->tc, p->cfg, Q, p->K, p->scores, (size_t)p->units * p->cfg.pot_size, N, M, p->units, p->status,
+        rc = tc_launch(p->tc, p->cfg, Q, p->K, cap_stats, p->scores, (size_t)p->units * p->cfg.pot_size, N, M, p->units, p->status,
                        p->stream, parts, &n_launch);
         p->launches += n_launch;
     } else {
-        rc = p->cfg.dtype == IPOT_F32 ? launch_simt<float>(p, Q, M, N) : launch_simt<__nv_bfloat16>(p, Q, M, N);
+        rc = p->cfg.dtype == IPOT_F32 ? launch_simt<float>(p, Q, cap_stats, M, N) : launch_simt<__nv_bfloat16>(p, Q, cap_stats, M, N);
     }
     if (rc != IPOT_OK) return rc;
     if (ev) IPOT_CUDA(cudaEventRecord(ev[2], p->stream));
@@ -162,12 +194,12 @@ int compact_slices(const ipot *p)
     return slices;
 }
 
-int run_cycle(ipot *p, const void *Q, int cap_rows, const float *aux)
+int run_cycle(ipot *p, const void *Q, const void *Kc, int cap_rows, const float *aux)
 {
     const int N = p->len, keep = p->cfg.keep, T = p->cfg.nuc_slots;
     int parts = 1;
     cudaEvent_t *ev = (p->profiling && p->ev_used < kProfSlots) ? p->ev[p->ev_used] : nullptr;
-    int rc = run_scoring(p, Q, cap_rows, aux, &parts);
+    int rc = run_scoring(p, Q, Kc, cap_rows, aux, &parts);
     if (rc != IPOT_OK) return rc;
     const size_t part_stride = (size_t)p->units * p->cfg.pot_size;
     select_kernel<<<p->units, kSelThreads, (size_t)N * 4, p->stream>>>(
@@ -239,10 +271,12 @@ int ipot_create_ex(const ipot_config_t *cfg, ipot_t **out)
     alloc((void **)&p->scores, score_elems * 4 * p->max_parts);
     alloc((void **)&p->summed, score_elems * 4);
     alloc((void **)&p->row_stats, (size_t)p->units * maxM * sizeof(float2));
+    alloc((void **)&p->cap_stats, (size_t)p->units * maxM * sizeof(float2));
     alloc((void **)&p->nuc_mask, (size_t)cfg->batch * cfg->pot_size);
     alloc((void **)&p->idx, (size_t)p->units * cfg->keep * 4);
     alloc((void **)&p->status, 16);
     alloc(&p->stage_q, (size_t)p->units * maxM * p->row_bytes);
+    alloc(&p->stage_kc, (size_t)p->units * cfg->max_cap_rows * p->row_bytes);
     alloc((void **)&p->stage_aux, (size_t)cfg->batch * cfg->pot_size * 4);
     if (ok) ok = cudaMemset(p->status, 0, 16) == cudaSuccess;
     if (!ok) {
@@ -256,6 +290,7 @@ int ipot_create_ex(const ipot_config_t *cfg, ipot_t **out)
          cudaFuncSetAttribute(cap_column_sums<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)simt_smem_bytes(256)) == cudaSuccess &&
          cudaFuncSetAttribute(cap_row_stats<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)simt_smem_bytes(256)) == cudaSuccess &&
          cudaFuncSetAttribute(cap_column_sums<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)simt_smem_bytes(256)) == cudaSuccess &&
+         cudaFuncSetAttribute(cap_self_stats_bf16, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)self_smem_bytes(256)) == cudaSuccess &&
          cudaFuncSetAttribute(nuc_mask_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 32768 * 4) == cudaSuccess &&
          cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 32768 * 4) == cudaSuccess;
     if (!ok) {
@@ -342,7 +377,7 @@ int ipot_score_and_compress(ipot_t *p, const void *Q, int cap_rows, const float 
     int rc = check_cycle_args(p, Q, cap_rows, aux, true);
     if (rc != IPOT_OK) return rc;
     if (!aligned16(Q) || (aux && (reinterpret_cast<uintptr_t>(aux) & 3u))) return IPOT_E_INVALID;
-    return run_cycle(p, Q, cap_rows, aux);
+    return run_cycle(p, Q, nullptr, cap_rows, aux);
 }
 
 int ipot_score_and_compress_host(ipot_t *p, const void *Q, int cap_rows, const float *aux, int32_t *idx_host)
@@ -352,20 +387,18 @@ int ipot_score_and_compress_host(ipot_t *p, const void *Q, int cap_rows, const f
     const size_t qbytes = (size_t)p->units * p->G * cap_rows * p->row_bytes;
     IPOT_CUDA(cudaMemcpyAsync(p->stage_q, Q, qbytes, cudaMemcpyHostToDevice, p->stream));
     if (aux) IPOT_CUDA(cudaMemcpyAsync(p->stage_aux, aux, (size_t)p->cfg.batch * p->len * 4, cudaMemcpyHostToDevice, p->stream));
-    rc = run_cycle(p, p->stage_q, cap_rows, aux ? p->stage_aux : nullptr);
+    rc = run_cycle(p, p->stage_q, nullptr, cap_rows, aux ? p->stage_aux : nullptr);
     if (rc != IPOT_OK) return rc;
     if (idx_host)
         IPOT_CUDA(cudaMemcpyAsync(idx_host, p->idx, (size_t)p->units * p->cfg.keep * 4, cudaMemcpyDeviceToHost, p->stream));
     return IPOT_OK;
 }
 
-int ipot_score_only(ipot_t *p, const void *Q, int cap_rows, const float *aux)
+namespace {
+int score_only(ipot *p, const void *Q, const void *Kc, int cap_rows, const float *aux)
 {
-    int rc = check_cycle_args(p, Q, cap_rows, aux, false);
-    if (rc != IPOT_OK) return rc;
-    if (!aligned16(Q)) return IPOT_E_INVALID;
     int parts = 1;
-    rc = run_scoring(p, Q, cap_rows, aux, &parts);
+    int rc = run_scoring(p, Q, Kc, cap_rows, aux, &parts);
     if (rc != IPOT_OK) return rc;
     if (parts > 1) {
         const size_t n = (size_t)p->units * p->len;
@@ -375,6 +408,47 @@ int ipot_score_only(ipot_t *p, const void *Q, int cap_rows, const float *aux)
         IPOT_CUDA(cudaGetLastError());
     }
     return IPOT_OK;
+}
+}  // namespace
+
+int ipot_score_only(ipot_t *p, const void *Q, int cap_rows, const float *aux)
+{
+    int rc = check_cycle_args(p, Q, cap_rows, aux, false);
+    if (rc != IPOT_OK) return rc;
+    if (!aligned16(Q)) return IPOT_E_INVALID;
+    return score_only(p, Q, nullptr, cap_rows, aux);
+}
+
+int ipot_score_and_compress_cap(ipot_t *p, const void *Q, const void *K_cap, int cap_rows, const float *aux)
+{
+    int rc = check_cycle_args(p, Q, cap_rows, aux, true);
+    if (rc != IPOT_OK) return rc;
+    if (!K_cap || !aligned16(Q) || !aligned16(K_cap) || (aux && (reinterpret_cast<uintptr_t>(aux) & 3u))) return IPOT_E_INVALID;
+    return run_cycle(p, Q, K_cap, cap_rows, aux);
+}
+
+int ipot_score_and_compress_cap_host(ipot_t *p, const void *Q, const void *K_cap, int cap_rows, const float *aux, int32_t *idx_host)
+{
+    int rc = check_cycle_args(p, Q, cap_rows, aux, true);
+    if (rc != IPOT_OK) return rc;
+    if (!K_cap) return IPOT_E_INVALID;
+    const size_t qbytes = (size_t)p->units * p->G * cap_rows * p->row_bytes, kcbytes = (size_t)p->units * cap_rows * p->row_bytes;
+    IPOT_CUDA(cudaMemcpyAsync(p->stage_q, Q, qbytes, cudaMemcpyHostToDevice, p->stream));
+    IPOT_CUDA(cudaMemcpyAsync(p->stage_kc, K_cap, kcbytes, cudaMemcpyHostToDevice, p->stream));
+    if (aux) IPOT_CUDA(cudaMemcpyAsync(p->stage_aux, aux, (size_t)p->cfg.batch * p->len * 4, cudaMemcpyHostToDevice, p->stream));
+    rc = run_cycle(p, p->stage_q, p->stage_kc, cap_rows, aux ? p->stage_aux : nullptr);
+    if (rc != IPOT_OK) return rc;
+    if (idx_host)
+        IPOT_CUDA(cudaMemcpyAsync(idx_host, p->idx, (size_t)p->units * p->cfg.keep * 4, cudaMemcpyDeviceToHost, p->stream));
+    return IPOT_OK;
+}
+
+int ipot_score_only_cap(ipot_t *p, const void *Q, const void *K_cap, int cap_rows, const float *aux)
+{
+    int rc = check_cycle_args(p, Q, cap_rows, aux, false);
+    if (rc != IPOT_OK) return rc;
+    if (!K_cap || !aligned16(Q) || !aligned16(K_cap)) return IPOT_E_INVALID;
+    return score_only(p, Q, K_cap, cap_rows, aux);
 }
 
 int ipot_view(ipot_t *p, void **K, void **V, int *len)
@@ -504,7 +578,7 @@ int noalloc_launch(const void *Q, const void *K, float *scores, float2 *stats, i
     IPOT_CUDA(cudaFuncSetAttribute(cap_column_sums<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)simt_smem_bytes(256)));
     const float scale_log2e = (float)(1.4426950408889634 / std::sqrt((double)d));
     dim3 g1((M + kSimtRows - 1) / kSimtRows, units), g2((N + kSimtKeys - 1) / kSimtKeys, units);
-    cap_row_stats<T><<<g1, kSimtThreads, smem, stream>>>((const T *)Q, (const T *)K, stats, M, N, d, k_unit_rows * d, scale_log2e);
+    cap_row_stats<T><<<g1, kSimtThreads, smem, stream>>>((const T *)Q, (const T *)K, stats, M, N, d, k_unit_rows * d, scale_log2e, nullptr, 0, 1);
     cap_column_sums<T><<<g2, kSimtThreads, smem, stream>>>((const T *)Q, (const T *)K, stats, scores, M, N, d, k_unit_rows * d, scale_log2e);
     IPOT_CUDA(cudaGetLastError());
     return IPOT_OK;

@@ -1,7 +1,10 @@
 // CaP scoring with plain fp32 FMAs (Sec. 3.3.1, Eq. 2): any supported shape,
 // f32 or bf16 storage.  Two launches per cycle:
 //   cap_row_stats  : per query row, the maximum logit and the reciprocal of the
-//                    softmax denominator over the N pot keys;
+//                    softmax denominator over the N pot keys;  the same kernel,
+//                    run over the CaP's own keys with a causal limit, gives the
+//                    share of the denominator that Appendix B's listing adds
+//                    (CaP queries also attend to the CaP keys before them);
 //   cap_column_sums: recomputes the logits per 64-key slab and adds
 //                    exp(s - max) / denominator over all query rows of the unit.
 // The M x N probability matrix lives only in registers.  Logits are kept in
@@ -79,11 +82,15 @@ __device__ __forceinline__ void merge_stats(float &m, float &l, float m2, float 
     l = a + b;
 }
 
-// grid (ceil(M / 32), units).  stats[unit][row] = (max logit in log2 units, 1 / sum_j 2^(x_j - max)).
+// grid (ceil(M / 32), units).  Row statistics over the keys Kpot[unit][0..N): (max logit in log2 units, sum_j 2^(x_j - max)).
+//   causal_P > 0 : row r only sees the keys 0 .. r % causal_P (the CaP keys up to the row's own position);
+//   extra        : if not NULL, (max, sum) pairs [unit][M] merged into the row's statistics first;
+//   reciprocal   : store 1 / sum instead of the sum (what cap_column_sums multiplies by).
 template <typename T>
 __global__ void __launch_bounds__(kSimtThreads)
 cap_row_stats(const T *__restrict__ Q, const T *__restrict__ Kpot, float2 *__restrict__ stats,
-              int M, int N, int d, size_t k_unit_stride, float scale_log2e)
+              int M, int N, int d, size_t k_unit_stride, float scale_log2e,
+              const float2 *__restrict__ extra, int causal_P, int reciprocal)
 {
     extern __shared__ __align__(16) float simt_sm[];
     float *Qs = simt_sm, *Ks = simt_sm + kSimtRows * (d + 4);
@@ -94,6 +101,9 @@ cap_row_stats(const T *__restrict__ Q, const T *__restrict__ Kpot, float2 *__res
 
     stage_rows(Qs, Qu, i0, kSimtRows, M, d);
     float m[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};
+    int lim[2];  // keys this thread's rows may see
+#pragma unroll
+    for (int a = 0; a < 2; ++a) lim[a] = causal_P > 0 ? min(N, (i0 + ty + 16 * a) % causal_P + 1) : N;
     for (int j0 = 0; j0 < N; j0 += kSimtKeys) {
         __syncthreads();
         stage_rows(Ks, Ku, j0, kSimtKeys, N, d);
@@ -106,13 +116,13 @@ cap_row_stats(const T *__restrict__ Q, const T *__restrict__ Kpot, float2 *__res
 #pragma unroll
             for (int b = 0; b < 4; ++b) {
                 acc[a][b] *= scale_log2e;
-                if (j0 + tx + 16 * b < N) tm = fmaxf(tm, acc[a][b]);
+                if (j0 + tx + 16 * b < lim[a]) tm = fmaxf(tm, acc[a][b]);
             }
             if (tm > -INFINITY) {
                 float tl = 0.f;
 #pragma unroll
                 for (int b = 0; b < 4; ++b)
-                    if (j0 + tx + 16 * b < N) tl += exp2f(acc[a][b] - tm);
+                    if (j0 + tx + 16 * b < lim[a]) tl += exp2f(acc[a][b] - tm);
                 merge_stats(m[a], l[a], tm, tl);
             }
         }
@@ -126,7 +136,13 @@ cap_row_stats(const T *__restrict__ Q, const T *__restrict__ Kpot, float2 *__res
             merge_stats(m[a], l[a], m2, l2);
         }
         const int row = i0 + ty + 16 * a;
-        if (tx == 0 && row < M) stats[(size_t)unit * M + row] = make_float2(m[a], 1.f / l[a]);
+        if (tx == 0 && row < M) {
+            if (extra) {
+                const float2 e = extra[(size_t)unit * M + row];
+                merge_stats(m[a], l[a], e.x, e.y);
+            }
+            stats[(size_t)unit * M + row] = make_float2(m[a], reciprocal ? 1.f / l[a] : l[a]);
+        }
     }
 }
 

@@ -21,7 +21,8 @@
 //            store whose sum carries the launch's sign as a "fresh" mark; then reads
 //            the row's statistics of all slabs of the item, re-reading until every
 //            one is fresh, and turns them into the row's global maximum m, its
-//            denominator l and the weights 2^(max_chunk - m) / l of the stored e values;
+//            denominator l (plus, when given, the share of the CaP's own keys) and the
+//            weights 2^(max_chunk - m) / l of the stored e values;
 //   pass 2   (the same 16 warps, one task behind: after pass 1 of task t+1 they
 //            finish task t, whose weights have arrived meanwhile)
 //            u_j = sum_i e_ij 2^(max_i - m_i) / l_i as a weighted column sum: the
@@ -73,6 +74,7 @@ struct TcParams {
     float *scores;        // partial array p (query rows 128p ...) at scores + p * part_stride, unit stride N
     size_t part_stride;
     float2 *stats;        // [items][slabs][128] (max in log2 units, sum * sign); all of the other sign or 0 at launch
+    const float2 *cap_stats;  // NULL, or [units][M] (max, sum) over the CaP's own keys that join every row's denominator
     float sign;           // +1 or -1: this launch's "fresh" mark
     int *status;
     int N, M, mtiles, slabs, tasks;
@@ -496,6 +498,9 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
             const int item = task / tasks_per_item, slab = task - item * tasks_per_item;
             const int mt = item % prm.mtiles;
             const uint32_t b = k & 1, ph = (k >> 1) & 1;
+            const bool row_valid = mt * kTcRows + row < prm.M;
+            float2 own = make_float2(-INFINITY, 0.f);  // the CaP keys' share of this row's denominator (Appendix B listing)
+            if (prm.cap_stats && row_valid) own = __ldg(&prm.cap_stats[(size_t)(item / prm.mtiles) * prm.M + mt * kTcRows + row]);
             mbar_wait(bar(kBarEReady + b), ph, ab, prm.status);
             // ---- merge the eight chunks of the row, publish the slab's statistics
             float cm[8];
@@ -540,7 +545,11 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                 for (int s = 0; s < 16; ++s) l = fmaf(fabsf(sv[s].y), ex2(sv[s].x - mb), l);
                 m = mb;
             }
-            const bool row_valid = mt * kTcRows + row < prm.M;
+            if (own.x > -INFINITY) {
+                const float mb = fmaxf(m, own.x);
+                l = fmaf(own.y, ex2(own.x - mb), l * ex2(m - mb));
+                m = mb;
+            }
             const float inv_l = row_valid ? 1.f / l : 0.f;
 #pragma unroll
             for (int i = 0; i < 8; ++i)
@@ -637,8 +646,8 @@ inline int tc_encode_rows(TcPlan &plan, CUtensorMap *map, const void *ptr, int r
 }
 
 // scores: partial array p (query rows 128 p ...) is written at scores + p * part_stride, unit stride N.
-inline int tc_launch(TcPlan &plan, const ipot_config_t &cfg, const void *Q, const void *K, float *scores, size_t part_stride,
-                     int N, int M, int units, int *status, cudaStream_t stream, int *parts, int *n_launch)
+inline int tc_launch(TcPlan &plan, const ipot_config_t &cfg, const void *Q, const void *K, const float2 *cap_stats, float *scores,
+                     size_t part_stride, int N, int M, int units, int *status, cudaStream_t stream, int *parts, int *n_launch)
 {
     if (!tc_applicable(plan, cfg, N, M)) return IPOT_E_INVALID;
     const int mtiles = (M + kTcRows - 1) / kTcRows;
@@ -646,7 +655,7 @@ inline int tc_launch(TcPlan &plan, const ipot_config_t &cfg, const void *Q, cons
     if (tc_encode_rows(plan, &mapQ, Q, M, units, (size_t)M, kTcRows) != IPOT_OK) return IPOT_E_CUDA;
     if (tc_encode_rows(plan, &mapK, K, N, units, (size_t)cfg.pot_size, kTcSlab) != IPOT_OK) return IPOT_E_CUDA;
     TcParams prm;
-    prm.scores = scores; prm.part_stride = part_stride; prm.stats = plan.stats; prm.status = status;
+    prm.scores = scores; prm.part_stride = part_stride; prm.stats = plan.stats; prm.cap_stats = cap_stats; prm.status = status;
     prm.N = N; prm.M = M; prm.mtiles = mtiles; prm.slabs = (N + kTcSlab - 1) / kTcSlab;
     const int items = units * mtiles;
     prm.tasks = items * prm.slabs;

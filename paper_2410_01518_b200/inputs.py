@@ -17,6 +17,7 @@ Layouts (all C-contiguous)
 ``K, V``  : ``[L][B][Hkv][n][d]``      pot rows of one chunk / one full pot
 ``Q``     : ``[L][B][Hq][P][d]``       catalyst-prompt (CaP) query rows
 ``aux``   : ``[B][N]`` float32         per-slot novelty (NuC) score, higher = more novel
+``K_cap`` : ``[L][B][Hkv][P][d]``      the CaP's own key rows (CaP-inclusive scoring only)
 
 Random streams are counter based (Philox): every tensor is keyed by
 ``(seed, config, tensor id, layer, cycle-or-chunk)`` so a subset of layers or
@@ -29,7 +30,7 @@ import numpy as np
 
 SEED_BASE = 0x1F1F0000
 
-_T_K, _T_V, _T_Q, _T_AUX, _T_MISC = 1, 2, 3, 4, 5
+_T_K, _T_V, _T_Q, _T_AUX, _T_MISC, _T_KCAP = 1, 2, 3, 4, 5, 6
 
 
 @dataclass(frozen=True)
@@ -167,6 +168,19 @@ def make_q(cfg: CcdConfig, cycle: int = 0, layers=None, cap_rows: int | None = N
         if cfg.recipe == "rope":
             q = _rope_rotate_half(q, np.arange(cfg.pot_size, cfg.pot_size + P))
         out.append(store(q, cfg.dtype))
+    return np.stack(out, axis=0)
+
+
+def make_kcap(cfg: CcdConfig, cycle: int = 0, layers=None, cap_rows: int | None = None) -> np.ndarray:
+    """K_cap[L][B][Hkv][P][d] in storage dtype: the key rows of the CaP positions."""
+    P = cfg.cap_rows if cap_rows is None else cap_rows
+    layers = range(cfg.layers) if layers is None else layers
+    out = []
+    for l in layers:
+        k = _normal(_gen(cfg.seed, _T_KCAP, l, cycle), (cfg.batch, cfg.Hkv, P, cfg.d))
+        if cfg.recipe == "rope":
+            k = _rope_rotate_half(k, np.arange(cfg.pot_size, cfg.pot_size + P))
+        out.append(store(k, cfg.dtype))
     return np.stack(out, axis=0)
 
 

@@ -28,6 +28,7 @@ SYMBOLS = [
     "ipot_score_and_compress", "ipot_score_and_compress_host", "ipot_score_only", "ipot_view",
     "ipot_last_indices", "ipot_last_scores", "ipot_sync_status", "ipot_set_profiling",
     "ipot_kernel_ms", "ipot_launch_count", "ipot_strerror", "ipot_cap_scores_noalloc",
+    "ipot_score_and_compress_cap", "ipot_score_only_cap", "ipot_score_and_compress_cap_host",
 ]
 
 
@@ -71,6 +72,9 @@ def lib() -> C.CDLL:
         L.ipot_score_and_compress.argtypes = [vp, vp, ip, vp]
         L.ipot_score_and_compress_host.argtypes = [vp, vp, ip, vp, vp]
         L.ipot_score_only.argtypes = [vp, vp, ip, vp]
+        L.ipot_score_and_compress_cap.argtypes = [vp, vp, vp, ip, vp]
+        L.ipot_score_only_cap.argtypes = [vp, vp, vp, ip, vp]
+        L.ipot_score_and_compress_cap_host.argtypes = [vp, vp, vp, ip, vp, vp]
         L.ipot_view.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(ip)]
         L.ipot_last_indices.argtypes = [vp, C.POINTER(vp)]
         L.ipot_last_scores.argtypes = [vp, C.POINTER(vp), C.POINTER(ip)]
@@ -161,6 +165,20 @@ def ipot_score_and_compress_host(h, Q_cap, cap_rows, aux_scores, idx_out=None) -
 
 def ipot_score_only(h, Q_cap, cap_rows, aux_scores=None) -> None:
     _check(lib().ipot_score_only(h, _ptr(Q_cap), cap_rows, _ptr(aux_scores)), "ipot_score_only")
+
+
+def ipot_score_and_compress_cap(h, Q_cap, K_cap, cap_rows, aux_scores) -> None:
+    _check(lib().ipot_score_and_compress_cap(h, _ptr(Q_cap), _ptr(K_cap), cap_rows, _ptr(aux_scores)),
+           "ipot_score_and_compress_cap")
+
+
+def ipot_score_and_compress_cap_host(h, Q_cap, K_cap, cap_rows, aux_scores, idx_out=None) -> None:
+    _check(lib().ipot_score_and_compress_cap_host(h, _ptr(Q_cap), _ptr(K_cap), cap_rows, _ptr(aux_scores), _ptr(idx_out)),
+           "ipot_score_and_compress_cap_host")
+
+
+def ipot_score_only_cap(h, Q_cap, K_cap, cap_rows, aux_scores=None) -> None:
+    _check(lib().ipot_score_only_cap(h, _ptr(Q_cap), _ptr(K_cap), cap_rows, _ptr(aux_scores)), "ipot_score_only_cap")
 
 
 def ipot_view(h):

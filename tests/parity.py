@@ -67,7 +67,11 @@ def gpu_cycle(cfg: inputs.CcdConfig, t: dict, scorer=ipot.IPOT_SCORER_AUTO, n=No
         Qd = to_dev(t["Q"], cfg.dtype)
         auxd = torch.from_numpy(np.ascontiguousarray(t["aux"][:, :n])).cuda()
         ipot.ipot_append_chunk(h, Kd, Vd, n)
-        ipot.ipot_score_and_compress(h, Qd, t["Q"].shape[3], auxd if cfg.nuc_slots > 0 else None)
+        if t.get("K_cap") is not None:  # Appendix B listing: the CaP's own keys join the softmax
+            ipot.ipot_score_and_compress_cap(h, Qd, to_dev(t["K_cap"], cfg.dtype), t["Q"].shape[3],
+                                             auxd if cfg.nuc_slots > 0 else None)
+        else:
+            ipot.ipot_score_and_compress(h, Qd, t["Q"].shape[3], auxd if cfg.nuc_slots > 0 else None)
         return read_results(h, cfg, n)
     finally:
         ipot.ipot_destroy(h)
@@ -101,7 +105,7 @@ def compare_cycle(cfg, t, gpu, units=None, n=None):
     Returns (units whose index list is identical to the checker's, units compared)."""
     n = cfg.pot_size if n is None else n
     K_in, V_in = t["K"][:, :, :, :n], t["V"][:, :, :, :n]
-    ref = oracle.cycle(t["Q"], K_in, V_in, t["aux"][:, :n], cfg.keep, cfg.nuc_slots, units=units)
+    ref = oracle.cycle(t["Q"], K_in, V_in, t["aux"][:, :n], cfg.keep, cfg.nuc_slots, units=units, K_cap=t.get("K_cap"))
     u, idx, K, V = gpu
     Kf, Vf = K_in.reshape(cfg.units, n, cfg.d), V_in.reshape(cfg.units, n, cfg.d)
     M = cfg.G * t["Q"].shape[3]

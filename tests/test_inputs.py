@@ -54,3 +54,12 @@ def test_outlier_channels_fixed_per_stream():
     s = inputs._outlier_scale(cfg, 0)
     assert set(np.unique(s).tolist()) <= {1.0, 8.0}
     assert (s == inputs._outlier_scale(cfg, 0)).all()
+
+
+def test_cap_key_rows_are_seeded_and_shaped():
+    cfg = inputs.small_config(cfg_id=130, layers=2, batch=2, Hq=4, Hkv=2, d=64, cap_rows=5, dtype="bf16")
+    a, b = inputs.make_kcap(cfg, 3), inputs.make_kcap(cfg, 3)
+    assert a.shape == (2, 2, 2, 5, 64) and a.dtype == np.uint16 and (a == b).all()
+    assert not (a == inputs.make_kcap(cfg, 4)).all()
+    assert (inputs.make_kcap(cfg, 3, layers=[1])[0] == a[1]).all()          # a layer subset is the same stream
+    assert not (a[:, :, :, :, :] == inputs.make_q(cfg, 3)[:, :, :2]).all()  # independent of the queries
