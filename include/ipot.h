@@ -104,7 +104,7 @@ int ipot_set_scorer(ipot_t *pot, int scorer);
 int ipot_reset(ipot_t *pot);
 
 /*
- * Sec. 3.2 ("filling the remaining cache space sequentially"): copy n_tokens
+ * Sec. 3.2 (the free part of the cache is filled in order): copy n_tokens
  * new rows of every unit behind the rows already in the pot; len += n_tokens.
  * K, V: device, [layers][batch][Hkv][n_tokens][d].
  * Errors: INVALID (NULL, misaligned, n_tokens <= 0), STATE (len + n_tokens >

@@ -6,7 +6,7 @@ imported by the CUDA library or its Python binding; only the tests, the smoke
 check and the benchmark's CPU-baseline leg call it.
 """
 from .ccd import (build, cap_scores, cap_scores_incl, cycle, gather, max_threads, nuc_top, select,
-                  set_threads, widen_storage)
+                  set_threads, token_novelty, widen_storage)
 
 __all__ = ["build", "cap_scores", "cap_scores_incl", "cycle", "gather", "max_threads", "nuc_top", "select",
-           "set_threads", "widen_storage"]
+           "set_threads", "token_novelty", "widen_storage"]

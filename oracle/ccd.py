@@ -33,10 +33,11 @@ def _load():
         lib.ora_cap_scores_incl.argtypes = [dp, dp, dp, C.c_int, C.c_int, C.c_int, C.c_int, dp, dp]
         lib.ora_cycle_cap.argtypes = [dp, dp, dp, bp, bp, dp, ip, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
                                       C.c_int, C.c_int, C.c_int, C.c_size_t, dp, ip, bp, bp]
+        lib.ora_token_novelty.argtypes = [dp, ip, C.c_long, C.c_int, dp]
         lib.ora_set_threads.argtypes = [C.c_int]
         lib.ora_max_threads.restype = C.c_int
         for f in (lib.ora_nuc_top, lib.ora_cap_scores, lib.ora_select, lib.ora_gather,
-                  lib.ora_cycle, lib.ora_set_threads, lib.ora_cap_scores_incl, lib.ora_cycle_cap):
+                  lib.ora_cycle, lib.ora_set_threads, lib.ora_cap_scores_incl, lib.ora_cycle_cap, lib.ora_token_novelty):
             f.restype = None
         _lib = lib
     return _lib
@@ -66,6 +67,17 @@ def set_threads(n: int) -> None:
 
 def max_threads() -> int:
     return int(_load().ora_max_threads())
+
+
+def token_novelty(logits, labels) -> np.ndarray:
+    """Eq. 3: logits [n][V] (float64), labels [n] -> -log softmax(logits)[label] per token [n]."""
+    z = _f64(logits)
+    lab = np.ascontiguousarray(labels, dtype=np.int32)
+    n, V = z.shape
+    assert lab.shape == (n,)
+    out = np.empty(n, dtype=np.float64)
+    _load().ora_token_novelty(_p(z, C.c_double), _p(lab, C.c_int), n, V, _p(out, C.c_double))
+    return out
 
 
 def nuc_top(aux, T: int) -> np.ndarray:

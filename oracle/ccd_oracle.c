@@ -7,7 +7,9 @@
  * check and the CPU-baseline leg of the benchmark use it.
  *
  * What each function follows:
- *   ora_nuc_top      Sec. 3.3.3: "first select the Top_T highest NuC scores"
+ *   ora_token_novelty  Sec. 3.3.2, Eq. 3 (the Appendix B listing computes it as a per-token
+ *                    cross-entropy without reduction): n_t = -log softmax(logits_t)[x_t]
+ *   ora_nuc_top      Sec. 3.3.3: the T slots with the highest NuC score are taken first
  *   ora_cap_scores   Sec. 3.3.1, Eq. 2: sum over the CaP query rows of the
  *                    self-attention probability towards every pot key
  *   ora_select       Sec. 3.3.3 + Appendix B "Combine NuC and CaP" / "Final
@@ -42,7 +44,8 @@
  * CaP-only special cases, byte-wise gather identities.  CaP-inclusive variant:
  * Q = 0 closed form G * sum_i 1/(N+i+1), masked library softmax over the N+P
  * columns, far-away CaP keys reduce it to ora_cap_scores, a later CaP key never
- * changes an earlier row.
+ * changes an earlier row.  Token novelty: uniform logits give log V, V = 2 is a
+ * softplus, a constant added to a row changes nothing, library cross-entropy.
  */
 #include <math.h>
 #include <stdint.h>
@@ -64,6 +67,24 @@ static int ora_cmp_int(const void *a, const void *b)
 {
     int x = *(const int *)a, y = *(const int *)b;
     return (x > y) - (x < y);
+}
+
+/*
+ * Eq. 3: novelty of token t = -log P(x_t | prefix) = log sum_v exp(z_tv) - z_t,label for the
+ * model's logits z ([n][V], row stride V).  A label outside [0, V) gives 0 (such a token is
+ * ignored, as a padding position would be).
+ */
+void ora_token_novelty(const double *logits, const int *labels, long n, int V, double *out)
+{
+    for (long t = 0; t < n; ++t) {
+        const double *z = logits + (size_t)t * V;
+        if (labels[t] < 0 || labels[t] >= V) { out[t] = 0.0; continue; }
+        double m = -INFINITY;
+        for (int v = 0; v < V; ++v) if (z[v] > m) m = z[v];
+        double Z = 0.0;
+        for (int v = 0; v < V; ++v) Z += exp(z[v] - m);
+        out[t] = (m + log(Z)) - z[labels[t]];
+    }
 }
 
 /* The T slots with the largest aux value (ties: lower slot first), returned ascending. */

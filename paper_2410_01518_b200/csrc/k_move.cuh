@@ -1,5 +1,5 @@
 // Row movers of the pot:
-//   append_kernel  : Sec. 3.2, "filling the remaining cache space sequentially";
+//   append_kernel  : Sec. 3.2 - new rows go into the free slots behind the survivors, in order;
 //   compact_kernel : Appendix B "KV-cache compression" - K'[r] = K[idx[r]],
 //                    V'[r] = V[idx[r]] - done in place.
 // Both move 16-byte vectors.

@@ -329,3 +329,32 @@ def test_cycle_with_cap_keys_wiring():
                 assert (out["K"][unit] == K[l, b, kv][out["idx"][unit]]).all()
     base = oracle.cycle(Q, K, V, aux, keep, T)
     assert not np.allclose(base["u"], out["u"])
+
+
+# ---------------------------------------------------------------- Eq. 3: token novelty
+def test_novelty_closed_forms():
+    V = 37
+    out = oracle.token_novelty(np.full((3, V), 1.25), [0, 5, V - 1])
+    np.testing.assert_allclose(out, np.log(V), rtol=1e-14)                  # uniform prediction
+    z = np.array([[0.3, -1.1], [2.0, 2.0], [-4.0, 6.0]])
+    lab = [0, 1, 0]
+    want = [np.log1p(np.exp(z[i, 1 - lab[i]] - z[i, lab[i]])) for i in range(3)]   # V = 2: a softplus
+    np.testing.assert_allclose(oracle.token_novelty(z, lab), want, rtol=1e-13)
+    z = np.zeros((2, 50)); z[0, 7] = 60.0; z[1, 7] = -60.0                  # certain / hopeless
+    out = oracle.token_novelty(z, [7, 7])
+    assert 0 <= out[0] < 1e-20 and abs(out[1] - (60.0 + np.log(49))) < 1e-12
+    assert (oracle.token_novelty(np.ones((2, 9)), [-100, 9]) == 0).all()    # ignored positions
+
+
+def test_novelty_is_the_library_cross_entropy():
+    torch = pytest.importorskip("torch")
+    from scipy.special import logsumexp
+    g = rnd(60)
+    z = g.standard_normal((40, 513)) * 4
+    lab = g.integers(0, 513, 40)
+    out = oracle.token_novelty(z, lab)
+    np.testing.assert_allclose(out, logsumexp(z, axis=1) - z[np.arange(40), lab], rtol=1e-12)
+    ce = torch.nn.functional.cross_entropy(torch.from_numpy(z), torch.from_numpy(lab), reduction="none")
+    np.testing.assert_allclose(out, ce.numpy(), rtol=1e-12)
+    np.testing.assert_allclose(oracle.token_novelty(z + 123.0, lab), out, rtol=1e-9, atol=1e-11)  # shift invariance
+    assert (out > 0).all()
