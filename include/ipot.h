@@ -171,6 +171,28 @@ int ipot_score_and_compress_cap_host(ipot_t *pot, const void *Q_cap_host, const 
                                      const float *aux_host, int32_t *idx_host);
 
 /*
+ * Token novelty, the quantity the NuC criterion ranks (Sec. 3.3.2, Eq. 3): for every new token the
+ * cross-entropy of the model's prediction, n = -log softmax(z)[x] = log sum_v exp(z_v) - z_x, from the
+ * logits z of the position that predicted the token and the token id x that followed.  The result can
+ * be written straight into the aux_scores array of the next ipot_score_and_compress call.
+ *   logits       : device, [batch][n_tokens] rows of `vocab` values, `row_stride` elements apart
+ *                  (row_stride >= vocab), of type logits_dtype (IPOT_BF16 or IPOT_F32; need not be the
+ *                  pot's type); rows that start on a 16-byte boundary are read with 16-byte loads,
+ *                  others element by element.  Caller-owned, read-only.
+ *   labels       : device, [batch][n_tokens] int32 token ids; a negative id marks an ignored position
+ *                  (novelty 0); an id >= vocab also gives 0 and raises the sticky status IPOT_E_BOUNDS.
+ *   aux_out      : device fp32; token t of stream b goes to aux_out[b * aux_stride + slot0 + t], i.e.
+ *                  slot0 is the pot fill before the chunk was appended; aux_stride >= slot0 + n_tokens.
+ * batch * n_tokens <= 65535.  Asynchronous on the pot's stream.  Uses a library-owned scratch of
+ * 8 * batch * n_tokens * ceil(vocab / 8192) bytes that is allocated on first use and when a call needs
+ * more (those calls synchronise the stream and may return IPOT_E_NOMEM); no other allocation.
+ * Errors: INVALID (NULL, sizes, alignment of the element type), NOMEM, CUDA.
+ */
+int ipot_nuc_scores(ipot_t *pot, const void *logits, int logits_dtype, long long row_stride,
+                    const int32_t *labels, int n_tokens, int vocab, float *aux_out, long long aux_stride,
+                    int slot0);
+
+/*
  * Borrowed device pointers to the pot ([layers][batch][Hkv][pot_size][d]) and
  * the current fill.  Rows >= len are undefined.  The pointers stay valid until
  * ipot_destroy(); their contents are final once the stream's queued work ran.

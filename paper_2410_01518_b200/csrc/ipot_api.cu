@@ -12,6 +12,7 @@
 #include "common.cuh"
 #include "k_cap_self.cuh"
 #include "k_move.cuh"
+#include "k_novelty.cuh"
 #include "k_score_simt.cuh"
 #include "k_score_tc.cuh"
 #include "k_select.cuh"
@@ -40,6 +41,8 @@ struct ipot {
     int *status;         // sticky device status word
     void *stage_q;       // device staging for the *_host calls
     void *stage_kc;
+    float2 *nov_partial;  // [tokens][segments] scratch of ipot_nuc_scores, grown on demand
+    size_t nov_capacity;
     float *stage_aux;
     // results of the last cycle
     int last_len_before;
@@ -86,7 +89,7 @@ void free_all(ipot *p)
     tc_plan_destroy(p->tc);
     cudaFree(p->K); cudaFree(p->V); cudaFree(p->scores); cudaFree(p->summed);
     cudaFree(p->row_stats); cudaFree(p->cap_stats); cudaFree(p->nuc_mask); cudaFree(p->idx); cudaFree(p->status);
-    cudaFree(p->stage_q); cudaFree(p->stage_kc); cudaFree(p->stage_aux);
+    cudaFree(p->stage_q); cudaFree(p->stage_kc); cudaFree(p->stage_aux); cudaFree(p->nov_partial);
     if (p->ev) {
         for (int i = 0; i < kProfSlots; ++i)
             for (auto &e : p->ev[i]) if (e) cudaEventDestroy(e);
@@ -224,6 +227,23 @@ int run_cycle(ipot *p, const void *Q, const void *Kc, int cap_rows, const float 
     return IPOT_OK;
 }
 
+}  // namespace
+
+namespace {
+template <typename T>
+int launch_novelty(ipot *p, const void *logits, size_t row_stride, const int32_t *labels, int n_tokens, int vocab,
+                   float *out, size_t out_stride, int slot0)
+{
+    const size_t rows = (size_t)p->cfg.batch * n_tokens;
+    const int segs = (vocab + kNovSegElems - 1) / kNovSegElems;
+    dim3 g1(segs, (unsigned)rows);
+    novelty_partial_kernel<T><<<g1, kNovThreads, 0, p->stream>>>((const T *)logits, row_stride, vocab, segs, p->nov_partial);
+    novelty_finish_kernel<T><<<(unsigned)((rows + kNovThreads - 1) / kNovThreads), kNovThreads, 0, p->stream>>>(
+        (const T *)logits, row_stride, vocab, segs, p->nov_partial, labels, rows, n_tokens, out, out_stride, slot0, p->status);
+    p->launches += 2;
+    IPOT_CUDA(cudaGetLastError());
+    return IPOT_OK;
+}
 }  // namespace
 
 extern "C" {
@@ -449,6 +469,35 @@ int ipot_score_only_cap(ipot_t *p, const void *Q, const void *K_cap, int cap_row
     if (rc != IPOT_OK) return rc;
     if (!K_cap || !aligned16(Q) || !aligned16(K_cap)) return IPOT_E_INVALID;
     return score_only(p, Q, K_cap, cap_rows, aux);
+}
+
+int ipot_nuc_scores(ipot_t *p, const void *logits, int logits_dtype, long long row_stride, const int32_t *labels,
+                    int n_tokens, int vocab, float *aux_out, long long aux_stride, int slot0)
+{
+    if (!p || !logits || !labels || !aux_out) return IPOT_E_INVALID;
+    if (logits_dtype != IPOT_BF16 && logits_dtype != IPOT_F32) return IPOT_E_INVALID;
+    if (n_tokens < 1 || n_tokens > 65535 / p->cfg.batch || vocab < 1 || row_stride < vocab) return IPOT_E_INVALID;
+    if (slot0 < 0 || aux_stride < (long long)slot0 + n_tokens) return IPOT_E_INVALID;
+    const size_t elem = logits_dtype == IPOT_F32 ? 4 : 2;
+    if ((reinterpret_cast<uintptr_t>(logits) % elem) || (reinterpret_cast<uintptr_t>(labels) & 3u) ||
+        (reinterpret_cast<uintptr_t>(aux_out) & 3u))
+        return IPOT_E_INVALID;
+    const size_t rows = (size_t)p->cfg.batch * n_tokens;
+    const size_t need = rows * ((vocab + kNovSegElems - 1) / kNovSegElems);
+    if (need > p->nov_capacity) {  // first use or a larger shape: the only allocation outside ipot_create
+        IPOT_CUDA(cudaStreamSynchronize(p->stream));
+        cudaFree(p->nov_partial);
+        p->nov_partial = nullptr;
+        p->nov_capacity = 0;
+        if (cudaMalloc((void **)&p->nov_partial, need * sizeof(float2)) != cudaSuccess) {
+            cudaGetLastError();
+            return IPOT_E_NOMEM;
+        }
+        p->nov_capacity = need;
+    }
+    return logits_dtype == IPOT_F32
+               ? launch_novelty<float>(p, logits, (size_t)row_stride, labels, n_tokens, vocab, aux_out, (size_t)aux_stride, slot0)
+               : launch_novelty<__nv_bfloat16>(p, logits, (size_t)row_stride, labels, n_tokens, vocab, aux_out, (size_t)aux_stride, slot0);
 }
 
 int ipot_view(ipot_t *p, void **K, void **V, int *len)

@@ -30,7 +30,7 @@ import numpy as np
 
 SEED_BASE = 0x1F1F0000
 
-_T_K, _T_V, _T_Q, _T_AUX, _T_MISC, _T_KCAP = 1, 2, 3, 4, 5, 6
+_T_K, _T_V, _T_Q, _T_AUX, _T_MISC, _T_KCAP, _T_LOGIT = 1, 2, 3, 4, 5, 6, 7
 
 
 @dataclass(frozen=True)
@@ -182,6 +182,22 @@ def make_kcap(cfg: CcdConfig, cycle: int = 0, layers=None, cap_rows: int | None 
             k = _rope_rotate_half(k, np.arange(cfg.pot_size, cfg.pot_size + P))
         out.append(store(k, cfg.dtype))
     return np.stack(out, axis=0)
+
+
+def make_logits(seed: int, rows: int, vocab: int, dtype: str, chunk: int = 0, ignored: float = 0.0):
+    """Stand-in for a language-model head over one chunk: (logits[rows][vocab] in storage dtype,
+    labels[rows] int32).  Logits ~ N(0, 2.5^2); the labels are uniform token ids; for about half of
+    the rows the label's logit is raised by U(0.6, 1.6) x (log(vocab) + 3) (tokens the model predicted
+    well: the log-sum-exp of the other logits is about log(vocab) + 3), so novelty spans near 0 to
+    above log(vocab).  A fraction ``ignored`` of the labels is -100 (padding)."""
+    g = _gen(seed, _T_LOGIT, 0, chunk)
+    z = g.standard_normal((rows, vocab), dtype=np.float32) * np.float32(2.5)
+    labels = g.integers(0, vocab, rows).astype(np.int32)
+    boost = np.where(g.random(rows) < 0.5, (0.6 + g.random(rows)) * (np.log(vocab) + 3.0), 0.0).astype(np.float32)
+    z[np.arange(rows), labels] += boost
+    if ignored > 0:
+        labels = np.where(g.random(rows) < ignored, np.int32(-100), labels).astype(np.int32)
+    return store(z, dtype), labels
 
 
 def _outlier_scale(cfg: CcdConfig, layer: int) -> np.ndarray:

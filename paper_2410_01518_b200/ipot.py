@@ -29,6 +29,7 @@ SYMBOLS = [
     "ipot_last_indices", "ipot_last_scores", "ipot_sync_status", "ipot_set_profiling",
     "ipot_kernel_ms", "ipot_launch_count", "ipot_strerror", "ipot_cap_scores_noalloc",
     "ipot_score_and_compress_cap", "ipot_score_only_cap", "ipot_score_and_compress_cap_host",
+    "ipot_nuc_scores",
 ]
 
 
@@ -75,6 +76,7 @@ def lib() -> C.CDLL:
         L.ipot_score_and_compress_cap.argtypes = [vp, vp, vp, ip, vp]
         L.ipot_score_only_cap.argtypes = [vp, vp, vp, ip, vp]
         L.ipot_score_and_compress_cap_host.argtypes = [vp, vp, vp, ip, vp, vp]
+        L.ipot_nuc_scores.argtypes = [vp, vp, ip, C.c_longlong, vp, ip, ip, vp, C.c_longlong, ip]
         L.ipot_view.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(ip)]
         L.ipot_last_indices.argtypes = [vp, C.POINTER(vp)]
         L.ipot_last_scores.argtypes = [vp, C.POINTER(vp), C.POINTER(ip)]
@@ -179,6 +181,11 @@ def ipot_score_and_compress_cap_host(h, Q_cap, K_cap, cap_rows, aux_scores, idx_
 
 def ipot_score_only_cap(h, Q_cap, K_cap, cap_rows, aux_scores=None) -> None:
     _check(lib().ipot_score_only_cap(h, _ptr(Q_cap), _ptr(K_cap), cap_rows, _ptr(aux_scores)), "ipot_score_only_cap")
+
+
+def ipot_nuc_scores(h, logits, logits_dtype, row_stride, labels, n_tokens, vocab, aux_out, aux_stride, slot0) -> None:
+    _check(lib().ipot_nuc_scores(h, _ptr(logits), logits_dtype, row_stride, _ptr(labels), n_tokens, vocab,
+                                 _ptr(aux_out), aux_stride, slot0), "ipot_nuc_scores")
 
 
 def ipot_view(h):

@@ -63,3 +63,14 @@ def test_cap_key_rows_are_seeded_and_shaped():
     assert not (a == inputs.make_kcap(cfg, 4)).all()
     assert (inputs.make_kcap(cfg, 3, layers=[1])[0] == a[1]).all()          # a layer subset is the same stream
     assert not (a[:, :, :, :, :] == inputs.make_q(cfg, 3)[:, :, :2]).all()  # independent of the queries
+
+
+def test_logits_recipe():
+    z, lab = inputs.make_logits(9, 200, 500, "bf16", chunk=2, ignored=0.1)
+    z2, lab2 = inputs.make_logits(9, 200, 500, "bf16", chunk=2, ignored=0.1)
+    assert z.shape == (200, 500) and z.dtype == np.uint16 and (z == z2).all() and (lab == lab2).all()
+    assert lab.dtype == np.int32 and ((lab == -100) | ((lab >= 0) & (lab < 500))).all() and (lab == -100).any()
+    assert not (inputs.make_logits(9, 200, 500, "bf16", chunk=3)[0] == z).all()
+    zf = inputs.widen(z, "bf16")
+    ok = lab >= 0
+    assert (zf[ok, lab[ok]] > 5).mean() > 0.3      # about half of the labels are well predicted
