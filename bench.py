@@ -30,6 +30,8 @@ sys.path.insert(0, ROOT)
 from paper_2410_01518_b200 import inputs  # noqa: E402
 
 WORKLOADS = {"cfg2": 2, "cfg3": 3, "cfg4": 4, "cfg5": 5}
+# the token-novelty producer alone (Eq. 3): (vocabulary, new tokens per step), bf16 logits, one stream
+NOVELTY_WORKLOADS = {"nuc32k": (32000, 2048), "nuc128k": (128256, 2048)}
 RING = 4  # distinct chunks / query sets cycled through
 
 
@@ -170,6 +172,124 @@ def run_reference(args, cfg):
     print(json.dumps(line))
 
 
+def run_novelty(args):
+    """The novelty producer alone: a step turns one chunk's logits into per-token novelty scores."""
+    V, n = NOVELTY_WORKLOADS[args.workload]
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    workload = f"token novelty of {n} new tokens over a {V}-word vocabulary (bf16 logits)"
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        import oracle
+        sample = 128
+        z, lab = inputs.make_logits(inputs.SEED_BASE + V, sample, V, "bf16", 0)
+        zw = inputs.widen(z, "bf16")
+        for _ in range(args.warmup):
+            oracle.token_novelty(zw[:8], lab[:8])
+        times = []
+        for _ in range(args.steps):
+            t0 = time.perf_counter()
+            oracle.token_novelty(zw, lab)
+            times.append(time.perf_counter() - t0)
+        ms = float(np.mean(times)) * 1e3 * n / sample
+        value = n * 1e3 / ms
+        print(json.dumps({
+            "impl": "reference", "metric": "nuc_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": 1,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": {"workload": workload},
+            "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": 1, "kind": "oracle",
+                             "sample": f"{sample} of {n} rows per step, extrapolated"},
+            "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2410_01518_b200 import ipot
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the compression path has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    ring = [inputs.make_logits(inputs.SEED_BASE + V, n, V, "bf16", c) for c in range(RING)]  # > L2 in total
+    dz = [torch.from_numpy(z.view(np.int16)).cuda().view(torch.bfloat16) for z, _ in ring]
+    dl = [torch.from_numpy(lab).cuda() for _, lab in ring]
+    hz = [torch.from_numpy(z.view(np.int16)).pin_memory() for z, _ in ring]
+    hl = [torch.from_numpy(lab).pin_memory() for _, lab in ring]
+    stage_z, stage_l = torch.empty_like(dz[0]), torch.empty_like(dl[0])
+    aux = torch.zeros((1, 2 * n), device="cuda")
+    aux_host = torch.empty((n,), dtype=torch.float32).pin_memory()
+    h = ipot.ipot_create_ex(2 * n, n, 1, 8, 8, 128, batch=1, dtype=ipot.IPOT_BF16, nuc_slots=n // 2, max_cap_rows=1)
+    stream = torch.cuda.current_stream()
+    ipot.ipot_set_stream(h, stream.cuda_stream)
+
+    def step_dev(i):
+        ipot.ipot_nuc_scores(h, dz[i % RING], ipot.IPOT_BF16, V, dl[i % RING], n, V, aux, 2 * n, n)
+
+    def step_host(i):
+        stage_z.view(torch.int16).copy_(hz[i % RING], non_blocking=True)
+        stage_l.copy_(hl[i % RING], non_blocking=True)
+        ipot.ipot_nuc_scores(h, stage_z, ipot.IPOT_BF16, V, stage_l, n, V, aux, 2 * n, n)
+        aux_host.copy_(aux[0, n:], non_blocking=True)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(step, steps, warmup, sampler=None):
+        for i in range(warmup):
+            step(i)
+        barrier()
+        if sampler:
+            sampler.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        l0 = ipot.ipot_launch_count(h)
+        e0.record(stream)
+        for i in range(steps):
+            step(warmup + i)
+        e1.record(stream)
+        barrier()
+        clocks = sampler.stop() if sampler else None
+        rate, ms_step = whole_job_rate(e0.elapsed_time(e1), steps, world, "cuda")
+        return rate * n, ms_step, ipot.ipot_launch_count(h) - l0, clocks
+
+    value, ms_step, launches, clocks = timed(step_dev, args.steps, args.warmup, ClockSampler(local))
+    e2e_value, _, _, _ = timed(step_host, max(3, min(args.steps, 50)), 3)
+    assert ipot.ipot_sync_status(h) == 0, "device status is not clean"
+    pk = peaks()
+    algo = n * V * 2 + n * 4 + n * 4   # logits once + labels + novelty out
+    roof = {"kernel": "novelty_partial_kernel", "bound": "hbm", "achieved": algo / (ms_step * 1e-3) / 1e9,
+            "peak": pk["hbm_gbs"], "unit": "GB/s", "peak_source": pk["source"], "traffic": None,
+            "note": "duration = the whole step (all launches of one call)"}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    line = {
+        "metric": "nuc_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": workload, "l2": "inputs_larger_than_l2", "ring": RING},
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": n * V * 2 + n * 4, "d2h_bytes_per_step": n * 4},
+        "gpu_launches": launches, "roofline": roof,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        sample = 256
+        zw = inputs.widen(ring[0][0][:sample], "bf16")
+        t0 = time.perf_counter()
+        oracle.token_novelty(zw, ring[0][1][:sample])
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": sample / dt, "unit": "tokens/s", "cores": 1, "kind": "oracle",
+                                "sample": f"{sample} of {n} rows of one step in {dt:.2f} s"}
+    if rank == 0:
+        print(json.dumps(line))
+    ipot.ipot_destroy(h)
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def config_dict(cfg, n_new, N, cap_keys=False):
     return {"workload": f"configs[{cfg.cfg_id - 1}] {cfg.name}: one CCD cycle per step "
                         f"(append {n_new} rows, distil {N} -> {cfg.keep})"
@@ -186,7 +306,7 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg3", choices=sorted(WORKLOADS))
+    ap.add_argument("--workload", default="cfg3", choices=sorted(WORKLOADS) + sorted(NOVELTY_WORKLOADS))
     ap.add_argument("--scorer", default="auto", choices=["auto", "simt", "tensor"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cap-keys", action="store_true",
@@ -194,6 +314,9 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (profiling small cases)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.workload in NOVELTY_WORKLOADS:
+        run_novelty(args)
+        return
     cfg = inputs.CONFIGS[WORKLOADS[args.workload]]
     if args.layers > 0:
         cfg = cfg.with_layers(args.layers)
