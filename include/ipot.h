@@ -184,8 +184,8 @@ int ipot_score_and_compress_cap_host(ipot_t *pot, const void *Q_cap_host, const 
  *   aux_out      : device fp32; token t of stream b goes to aux_out[b * aux_stride + slot0 + t], i.e.
  *                  slot0 is the pot fill before the chunk was appended; aux_stride >= slot0 + n_tokens.
  * batch * n_tokens <= 65535.  Asynchronous on the pot's stream.  Uses a library-owned scratch of
- * 8 * batch * n_tokens * ceil(vocab / 8192) bytes that is allocated on first use and when a call needs
- * more (those calls synchronise the stream and may return IPOT_E_NOMEM); no other allocation.
+ * 256 KiB + 8 * batch * n_tokens * ceil(vocab / 8192) bytes that is allocated on first use and when a
+ * call needs more (those calls synchronise the stream and may return IPOT_E_NOMEM); no other allocation.
  * Errors: INVALID (NULL, sizes, alignment of the element type), NOMEM, CUDA.
  */
 int ipot_nuc_scores(ipot_t *pot, const void *logits, int logits_dtype, long long row_stride,

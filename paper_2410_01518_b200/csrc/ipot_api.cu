@@ -41,8 +41,9 @@ struct ipot {
     int *status;         // sticky device status word
     void *stage_q;       // device staging for the *_host calls
     void *stage_kc;
-    float2 *nov_partial;  // [tokens][segments] scratch of ipot_nuc_scores, grown on demand
-    size_t nov_capacity;
+    char *nov_scratch;   // scratch of ipot_nuc_scores, grown on demand: 65536 row counters (always zero between
+                         // calls), then [tokens][segments] float2
+    size_t nov_capacity;  // float2 entries behind the counters
     float *stage_aux;
     // results of the last cycle
     int last_len_before;
@@ -59,6 +60,7 @@ struct ipot {
 namespace {
 
 constexpr int kProfSlots = 2048;
+constexpr size_t kNovCounterBytes = (size_t)(kNovMaxRows + 1) * sizeof(int);
 
 #define IPOT_CUDA(call)                                                             \
     do {                                                                            \
@@ -89,7 +91,7 @@ void free_all(ipot *p)
     tc_plan_destroy(p->tc);
     cudaFree(p->K); cudaFree(p->V); cudaFree(p->scores); cudaFree(p->summed);
     cudaFree(p->row_stats); cudaFree(p->cap_stats); cudaFree(p->nuc_mask); cudaFree(p->idx); cudaFree(p->status);
-    cudaFree(p->stage_q); cudaFree(p->stage_kc); cudaFree(p->stage_aux); cudaFree(p->nov_partial);
+    cudaFree(p->stage_q); cudaFree(p->stage_kc); cudaFree(p->stage_aux); cudaFree(p->nov_scratch);
     if (p->ev) {
         for (int i = 0; i < kProfSlots; ++i)
             for (auto &e : p->ev[i]) if (e) cudaEventDestroy(e);
@@ -236,11 +238,12 @@ int launch_novelty(ipot *p, const void *logits, size_t row_stride, const int32_t
 {
     const size_t rows = (size_t)p->cfg.batch * n_tokens;
     const int segs = (vocab + kNovSegElems - 1) / kNovSegElems;
-    dim3 g1(segs, (unsigned)rows);
-    novelty_partial_kernel<T><<<g1, kNovThreads, 0, p->stream>>>((const T *)logits, row_stride, vocab, segs, p->nov_partial);
-    novelty_finish_kernel<T><<<(unsigned)((rows + kNovThreads - 1) / kNovThreads), kNovThreads, 0, p->stream>>>(
-        (const T *)logits, row_stride, vocab, segs, p->nov_partial, labels, rows, n_tokens, out, out_stride, slot0, p->status);
-    p->launches += 2;
+    int *counters = reinterpret_cast<int *>(p->nov_scratch);
+    float2 *partial = reinterpret_cast<float2 *>(p->nov_scratch + kNovCounterBytes);
+    dim3 grid(segs, (unsigned)rows);
+    novelty_kernel<T><<<grid, kNovThreads, 0, p->stream>>>((const T *)logits, row_stride, vocab, segs, partial, counters, labels,
+                                                           n_tokens, out, out_stride, slot0, p->status);
+    p->launches += 1;
     IPOT_CUDA(cudaGetLastError());
     return IPOT_OK;
 }
@@ -476,7 +479,7 @@ int ipot_nuc_scores(ipot_t *p, const void *logits, int logits_dtype, long long r
 {
     if (!p || !logits || !labels || !aux_out) return IPOT_E_INVALID;
     if (logits_dtype != IPOT_BF16 && logits_dtype != IPOT_F32) return IPOT_E_INVALID;
-    if (n_tokens < 1 || n_tokens > 65535 / p->cfg.batch || vocab < 1 || row_stride < vocab) return IPOT_E_INVALID;
+    if (n_tokens < 1 || n_tokens > kNovMaxRows / p->cfg.batch || vocab < 1 || row_stride < vocab) return IPOT_E_INVALID;
     if (slot0 < 0 || aux_stride < (long long)slot0 + n_tokens) return IPOT_E_INVALID;
     const size_t elem = logits_dtype == IPOT_F32 ? 4 : 2;
     if ((reinterpret_cast<uintptr_t>(logits) % elem) || (reinterpret_cast<uintptr_t>(labels) & 3u) ||
@@ -484,15 +487,16 @@ int ipot_nuc_scores(ipot_t *p, const void *logits, int logits_dtype, long long r
         return IPOT_E_INVALID;
     const size_t rows = (size_t)p->cfg.batch * n_tokens;
     const size_t need = rows * ((vocab + kNovSegElems - 1) / kNovSegElems);
-    if (need > p->nov_capacity) {  // first use or a larger shape: the only allocation outside ipot_create
+    if (!p->nov_scratch || need > p->nov_capacity) {  // first use or a larger shape: the only allocation outside ipot_create
         IPOT_CUDA(cudaStreamSynchronize(p->stream));
-        cudaFree(p->nov_partial);
-        p->nov_partial = nullptr;
+        cudaFree(p->nov_scratch);
+        p->nov_scratch = nullptr;
         p->nov_capacity = 0;
-        if (cudaMalloc((void **)&p->nov_partial, need * sizeof(float2)) != cudaSuccess) {
+        if (cudaMalloc((void **)&p->nov_scratch, kNovCounterBytes + need * sizeof(float2)) != cudaSuccess) {
             cudaGetLastError();
             return IPOT_E_NOMEM;
         }
+        IPOT_CUDA(cudaMemsetAsync(p->nov_scratch, 0, kNovCounterBytes, p->stream));
         p->nov_capacity = need;
     }
     return logits_dtype == IPOT_F32
