@@ -15,7 +15,7 @@ _lib = None
 def build(force: bool = False) -> str:
     """Compile the checker with gcc (-O2, OpenMP).  Returns the library path."""
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
-        subprocess.check_call(["gcc", "-O2", "-fopenmp", "-shared", "-fPIC", "-o", _LIB, _SRC, "-lm"])
+        subprocess.check_call(["gcc", "-O2", "-ffp-contract=off", "-fopenmp", "-shared", "-fPIC", "-o", _LIB, _SRC, "-lm"])
     return _LIB
 
 
@@ -34,10 +34,11 @@ def _load():
         lib.ora_cycle_cap.argtypes = [dp, dp, dp, bp, bp, dp, ip, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
                                       C.c_int, C.c_int, C.c_int, C.c_size_t, dp, ip, bp, bp]
         lib.ora_token_novelty.argtypes = [dp, ip, C.c_long, C.c_int, dp]
+        lib.ora_rope_rows.argtypes = [C.c_void_p, C.c_void_p, ip, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_int]
         lib.ora_set_threads.argtypes = [C.c_int]
         lib.ora_max_threads.restype = C.c_int
         for f in (lib.ora_nuc_top, lib.ora_cap_scores, lib.ora_select, lib.ora_gather,
-                  lib.ora_cycle, lib.ora_set_threads, lib.ora_cap_scores_incl, lib.ora_cycle_cap, lib.ora_token_novelty):
+                  lib.ora_cycle, lib.ora_set_threads, lib.ora_cap_scores_incl, lib.ora_cycle_cap, lib.ora_token_novelty, lib.ora_rope_rows):
             f.restype = None
         _lib = lib
     return _lib
@@ -67,6 +68,25 @@ def set_threads(n: int) -> None:
 
 def max_threads() -> int:
     return int(_load().ora_max_threads())
+
+
+def rope_rows(rows, pos, cos_t, sin_t, interleaved: bool = False) -> np.ndarray:
+    """Sec. 3.4: rotary embedding of rows [..., n, d] (storage dtype: float32 or uint16 bf16 bits) at positions
+    pos [n] with cos/sin tables [positions][d/2] of the same storage dtype; every leading index uses the same
+    positions.  Returns the rotated rows in the storage dtype."""
+    rows = np.ascontiguousarray(rows)
+    cos_t, sin_t = np.ascontiguousarray(cos_t), np.ascontiguousarray(sin_t)
+    assert rows.dtype in (np.float32, np.uint16) and cos_t.dtype == rows.dtype and sin_t.dtype == rows.dtype
+    n, d = rows.shape[-2], rows.shape[-1]
+    pos = np.ascontiguousarray(pos, dtype=np.int32)
+    assert pos.shape == (n,) and d % 2 == 0 and cos_t.shape == sin_t.shape and cos_t.shape[1] == d // 2
+    assert pos.min(initial=0) >= 0 and pos.max(initial=0) < cos_t.shape[0]
+    out = np.empty_like(rows)
+    flat_in, flat_out = rows.reshape(-1, n, d), out.reshape(-1, n, d)
+    for i in range(flat_in.shape[0]):
+        _load().ora_rope_rows(flat_in[i].ctypes.data, flat_out[i].ctypes.data, _p(pos, C.c_int), n, d,
+                              int(rows.dtype == np.float32), cos_t.ctypes.data, sin_t.ctypes.data, int(interleaved))
+    return out
 
 
 def token_novelty(logits, labels) -> np.ndarray:
@@ -136,7 +156,7 @@ def gather(rows: np.ndarray, idx) -> np.ndarray:
     return out
 
 
-def cycle(Q, K, V, aux, keep: int, T: int, units=None, with_kv: bool = True, K_cap=None):
+def cycle(Q, K, V, aux, keep: int, T: int, units=None, with_kv: bool = True, K_cap=None, rope=None):
     """One CCD cycle over all (or the listed) units.
 
     Q [L][B][Hq][P][d], K, V [L][B][Hkv][N][d] in storage dtype (float32 or
@@ -144,6 +164,9 @@ def cycle(Q, K, V, aux, keep: int, T: int, units=None, with_kv: bool = True, K_c
     ``(l*B + b)*Hkv + g``.  Returns a dict with ``units``, ``u`` [n][N],
     ``idx`` [n][keep] and, if ``with_kv``, the compacted ``K``, ``V`` [n][keep][d].
     With ``K_cap`` [L][B][Hkv][P][d] the scores are the CaP-inclusive ones.
+    With ``rope = (cos_t, sin_t, interleaved)`` K holds keys without rotary embedding: the scores use the keys
+    rotated at their slot number 0..N-1 (Sec. 3.4), the gather moves the unrotated rows, and ``K_rot``
+    [n][keep][d] is the compacted pot rotated at the new slot numbers 0..keep-1.
     """
     L, B, Hq, P, d = Q.shape
     Hkv, N = K.shape[2], K.shape[3]
@@ -160,7 +183,7 @@ def cycle(Q, K, V, aux, keep: int, T: int, units=None, with_kv: bool = True, K_c
     Ks = np.ascontiguousarray(Kf[units])
     Vs = np.ascontiguousarray(Vf[units])
     Qd = widen_storage(Qf[units])
-    Kd = widen_storage(Ks)
+    Kd = widen_storage(Ks if rope is None else rope_rows(Ks, np.arange(N), rope[0], rope[1], rope[2]))
     Kcd = None
     if K_cap is not None:
         assert K_cap.shape == (L, B, Hkv, P, d)
@@ -179,4 +202,7 @@ def cycle(Q, K, V, aux, keep: int, T: int, units=None, with_kv: bool = True, K_c
         Ks.ctypes.data_as(bp), Vs.ctypes.data_as(bp), _p(auxd, C.c_double), _p(stream_of, C.c_int),
         n, B, M, P, d, N, keep, T, rb, _p(u, C.c_double), _p(idx, C.c_int),
         Ko.ctypes.data_as(bp) if with_kv else None, Vo.ctypes.data_as(bp) if with_kv else None)
-    return {"units": units, "u": u, "idx": idx, "K": Ko, "V": Vo}
+    out = {"units": units, "u": u, "idx": idx, "K": Ko, "V": Vo}
+    if rope is not None and with_kv:
+        out["K_rot"] = rope_rows(Ko, np.arange(keep), rope[0], rope[1], rope[2])
+    return out

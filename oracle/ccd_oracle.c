@@ -21,6 +21,8 @@
  *                    queries attend to the pot keys AND, causally, to the CaP's
  *                    own keys; the CaP columns are then cut away, so they only
  *                    take probability mass from the pot columns
+ *   ora_rope_rows    Sec. 3.4 (CR-RoPE): keys are kept without rotary embedding and get it
+ *                    at their position inside the pot, 0 .. len-1
  *   ora_cycle        the four steps over every (layer, stream, kv-head) unit
  *   ora_cycle_cap    the same with the CaP-inclusive scores
  *
@@ -33,7 +35,14 @@
  *   - the CaP top-(|C|-T) is taken among slots not already taken by NuC, so
  *     exactly |C| slots survive;
  *   - ties: the lower slot index wins, in both rankings;
- *   - survivors keep their original order (ascending slot index).
+ *   - survivors keep their original order (ascending slot index);
+ *   - CR-RoPE: the paper gives no rotary details.  The caller supplies cos/sin per (position,
+ *     frequency) in the storage type; channel pairs are (c, c + d/2) ("half") or (2c, 2c + 1)
+ *     ("interleaved"); the rotation is evaluated in single precision exactly as
+ *     lo' = fma(lo, cos, -(hi * sin)), hi' = fma(hi, cos, lo * sin) and rounded once to the
+ *     storage type (nearest even).  Rounding to bf16 is a quantisation, so both the checker
+ *     and the CUDA path take it from the same single-precision expression; everything after
+ *     it (the scores) is double precision here.
  *
  *   - CaP-inclusive variant: CaP row i (0-based, within its query head) sees the
  *     CaP keys 0..i of its KV head (causal mask), all of them after every pot key;
@@ -46,6 +55,9 @@
  * columns, far-away CaP keys reduce it to ora_cap_scores, a later CaP key never
  * changes an earlier row.  Token novelty: uniform logits give log V, V = 2 is a
  * softplus, a constant added to a row changes nothing, library cross-entropy.
+ * Rotary rows: position 0 is the identity, exact small cases, complex multiplication in
+ * double precision, pair norms, the score of a rotated query and key depends on the
+ * position difference only, the two pairings are one channel permutation apart.
  */
 #include <math.h>
 #include <stdint.h>
@@ -161,6 +173,58 @@ void ora_cap_scores_incl(const double *Q, const double *K, const double *Kc, int
         if (pot_mass) pot_mass[r] = pm;
     }
     free(s);
+}
+
+/* ---- storage <-> float (bf16 = upper half of a float, rounded to nearest even) ---- */
+static float ora_bf16_to_float(uint16_t b)
+{
+    uint32_t w = (uint32_t)b << 16;
+    float f;
+    memcpy(&f, &w, 4);
+    return f;
+}
+
+static uint16_t ora_float_to_bf16(float f)
+{
+    uint32_t w;
+    memcpy(&w, &f, 4);
+    w += 0x7FFFu + ((w >> 16) & 1u);
+    return (uint16_t)(w >> 16);
+}
+
+static float ora_load(const void *p, size_t i, int is_f32)
+{
+    return is_f32 ? ((const float *)p)[i] : ora_bf16_to_float(((const uint16_t *)p)[i]);
+}
+
+static void ora_store(void *p, size_t i, int is_f32, float v)
+{
+    if (is_f32) ((float *)p)[i] = v;
+    else ((uint16_t *)p)[i] = ora_float_to_bf16(v);
+}
+
+/*
+ * Sec. 3.4: rotary embedding of n rows of d channels; row r gets position pos[r].  cos_t and
+ * sin_t are [positions][d/2] tables in the storage type.  interleaved = 0 pairs channel c with
+ * c + d/2, 1 pairs 2c with 2c + 1; frequency index c in both.  in and out may not overlap.
+ */
+void ora_rope_rows(const void *in, void *out, const int *pos, int n, int d, int is_f32,
+                   const void *cos_t, const void *sin_t, int interleaved)
+{
+    const int half = d / 2;
+    for (int r = 0; r < n; ++r) {
+        for (int c = 0; c < half; ++c) {
+            const size_t ilo = (size_t)r * d + (interleaved ? 2 * c : c);
+            const size_t ihi = (size_t)r * d + (interleaved ? 2 * c + 1 : c + half);
+            const float lo = ora_load(in, ilo, is_f32), hi = ora_load(in, ihi, is_f32);
+            const float cs = ora_load(cos_t, (size_t)pos[r] * half + c, is_f32);
+            const float sn = ora_load(sin_t, (size_t)pos[r] * half + c, is_f32);
+            volatile float t1 = hi * sn;   /* volatile: each product is rounded on its own */
+            volatile float t2 = lo * sn;
+            ora_store(out, ilo, is_f32, fmaf(lo, cs, -t1));
+            ora_store(out, ihi, is_f32, fmaf(hi, cs, t2));
+        }
+    }
 }
 
 /*

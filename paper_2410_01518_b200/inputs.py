@@ -151,6 +151,16 @@ def _rope_rotate_half(x: np.ndarray, pos: np.ndarray, base: float = 10000.0) -> 
     return out.astype(np.float32)
 
 
+def make_rope_table(positions: int, d: int, dtype: str, base: float = 10000.0):
+    """The caller's side of CR-RoPE: cos and sin of ``pos * base**(-c / (d/2))`` for pos < positions and
+    frequency c < d/2, evaluated in float64 and stored in the pot's storage dtype.  Returns (cos, sin),
+    each [positions][d/2]."""
+    half = d // 2
+    inv = base ** (-np.arange(half, dtype=np.float64) / half)
+    ang = np.arange(positions, dtype=np.float64)[:, None] * inv[None, :]
+    return store(np.cos(ang).astype(np.float32), dtype), store(np.sin(ang).astype(np.float32), dtype)
+
+
 def make_aux(cfg: CcdConfig, cycle: int = 0, n: int | None = None) -> np.ndarray:
     """aux[B][n] ~ U(0,1), float32."""
     n = cfg.pot_size if n is None else n

@@ -358,3 +358,95 @@ def test_novelty_is_the_library_cross_entropy():
     np.testing.assert_allclose(out, ce.numpy(), rtol=1e-12)
     np.testing.assert_allclose(oracle.token_novelty(z + 123.0, lab), out, rtol=1e-9, atol=1e-11)  # shift invariance
     assert (out > 0).all()
+
+
+# ---------------------------------------------------------------- Sec. 3.4: rotary embedding at pot positions
+def _tables(positions, d, dtype="f32"):
+    from paper_2410_01518_b200 import inputs
+    return inputs.make_rope_table(positions, d, dtype)
+
+
+def test_rope_exact_small_cases_and_identity():
+    x = np.array([[1, 2, 3, 4]], dtype=np.float32)
+    c = np.array([[1, 1], [0.5, 0.5], [0, 0]], dtype=np.float32)
+    s = np.array([[0, 0], [0.5, 0.5], [1, 1]], dtype=np.float32)
+    assert (oracle.rope_rows(x, [0], c, s) == x).all()                                  # angle 0
+    assert (oracle.rope_rows(x, [1], c, s) == [[-1, -1, 2, 3]]).all()                   # pairs (1,3), (2,4)
+    assert (oracle.rope_rows(x, [1], c, s, True) == [[-0.5, 1.5, -0.5, 3.5]]).all()     # pairs (1,2), (3,4)
+    assert (oracle.rope_rows(x, [2], c, s) == [[-3, -4, 1, 2]]).all()                   # quarter turn
+    cos_t, sin_t = _tables(16, 8)
+    g = rnd(70)
+    rows = g.standard_normal((3, 5, 8)).astype(np.float32)
+    out = oracle.rope_rows(rows, [0, 0, 0, 0, 0], cos_t, sin_t)
+    assert (out == rows).all()                                                          # position 0 everywhere
+
+
+def test_rope_is_complex_multiplication():
+    g = rnd(71)
+    d, n = 16, 40
+    cos_t, sin_t = _tables(64, d)
+    rows = g.standard_normal((n, d)).astype(np.float32)
+    pos = g.integers(0, 64, n)
+    out = oracle.rope_rows(rows, pos, cos_t, sin_t).astype(np.float64)
+    z = rows[:, :d // 2].astype(np.float64) + 1j * rows[:, d // 2:].astype(np.float64)
+    w = z * (cos_t[pos].astype(np.float64) + 1j * sin_t[pos].astype(np.float64))
+    np.testing.assert_allclose(out[:, :d // 2], w.real, rtol=0, atol=2e-6)
+    np.testing.assert_allclose(out[:, d // 2:], w.imag, rtol=0, atol=2e-6)
+    # pair norms survive the rotation (up to the table's rounding)
+    np.testing.assert_allclose(out[:, :d // 2] ** 2 + out[:, d // 2:] ** 2, np.abs(z) ** 2, rtol=1e-5)
+
+
+def test_rope_scores_depend_on_the_position_difference():
+    g = rnd(72)
+    d = 32
+    cos_t, sin_t = _tables(200, d)
+    q = g.standard_normal((1, d)).astype(np.float32)
+    k = g.standard_normal((1, d)).astype(np.float32)
+    dots = [float(oracle.rope_rows(q, [m], cos_t, sin_t).astype(np.float64)[0]
+                  @ oracle.rope_rows(k, [m - 17], cos_t, sin_t).astype(np.float64)[0]) for m in (17, 60, 199)]
+    assert max(dots) - min(dots) < 1e-4 * max(1.0, abs(dots[0]))
+    other = float(oracle.rope_rows(q, [60], cos_t, sin_t).astype(np.float64)[0]
+                  @ oracle.rope_rows(k, [60 - 18], cos_t, sin_t).astype(np.float64)[0])
+    assert abs(other - dots[0]) > 1e-3                                                  # and on nothing less
+
+
+def test_rope_pairings_are_a_channel_permutation_apart_and_bf16_rounds_once():
+    g = rnd(73)
+    d, n = 12, 9
+    rows = g.standard_normal((n, d)).astype(np.float32)
+    cos_t, sin_t = _tables(32, d)
+    pos = g.integers(0, 32, n)
+    # interleaved channels 2c, 2c + 1 hold what the half layout keeps in channels c, c + d/2
+    inter_in = np.empty_like(rows)
+    inter_in[:, 0::2], inter_in[:, 1::2] = rows[:, :d // 2], rows[:, d // 2:]
+    inter = oracle.rope_rows(inter_in, pos, cos_t, sin_t, True)
+    ref = oracle.rope_rows(rows, pos, cos_t, sin_t, False)
+    assert (inter[:, 0::2] == ref[:, :d // 2]).all() and (inter[:, 1::2] == ref[:, d // 2:]).all()
+    # bf16 storage: the float32 result rounded once to nearest even
+    from paper_2410_01518_b200 import inputs
+    rb, cb, sb = inputs.store(rows, "bf16"), *inputs.make_rope_table(32, d, "bf16")
+    got = oracle.rope_rows(rb, pos, cb, sb)
+    f = oracle.rope_rows(inputs.widen(rb, "bf16").astype(np.float32), pos, inputs.widen(cb, "bf16").astype(np.float32),
+                         inputs.widen(sb, "bf16").astype(np.float32))
+    assert (got == inputs.store(f, "bf16")).all()
+
+
+def test_cycle_with_rope_scores_rotated_keys_and_moves_unrotated_rows():
+    from paper_2410_01518_b200 import inputs
+    g = rnd(74)
+    L, B, Hq, Hkv, P, d, N, keep, T = 1, 2, 4, 2, 3, 8, 20, 9, 4
+    Q = g.standard_normal((L, B, Hq, P, d)).astype(np.float32)
+    K = g.standard_normal((L, B, Hkv, N, d)).astype(np.float32)
+    V = g.standard_normal((L, B, Hkv, N, d)).astype(np.float32)
+    aux = g.random((B, N)).astype(np.float32)
+    cos_t, sin_t = inputs.make_rope_table(N, d, "f32")
+    out = oracle.cycle(Q, K, V, aux, keep, T, rope=(cos_t, sin_t, False))
+    Kr = oracle.rope_rows(K, np.arange(N), cos_t, sin_t)
+    plain = oracle.cycle(Q, Kr, V, aux, keep, T)
+    np.testing.assert_array_equal(out["u"], plain["u"])
+    assert (out["idx"] == plain["idx"]).all()
+    for unit in range(L * B * Hkv):
+        src = K.reshape(-1, N, d)[unit][out["idx"][unit]]
+        assert (out["K"][unit] == src).all()                                           # unrotated rows move
+        assert (out["K_rot"][unit] == oracle.rope_rows(src, np.arange(keep), cos_t, sin_t)).all()   # new positions
+    assert not np.allclose(out["u"], oracle.cycle(Q, K, V, aux, keep, T)["u"])
