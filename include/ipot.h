@@ -57,6 +57,12 @@ enum {
 
 enum { IPOT_BF16 = 0, IPOT_F32 = 1 };
 
+/* Channel pairing of the rotary embedding (ipot_enable_rope). */
+enum {
+    IPOT_ROPE_HALF = 1,        /* channel c with c + d/2 */
+    IPOT_ROPE_INTERLEAVED = 2  /* channel 2c with 2c + 1 */
+};
+
 /* Which scoring kernel ipot_score_and_compress() uses. */
 enum {
     IPOT_SCORER_AUTO = 0,   /* tensor-core kernel when the shape allows it, else the SIMT kernel */
@@ -191,6 +197,32 @@ int ipot_score_and_compress_cap_host(ipot_t *pot, const void *Q_cap_host, const 
 int ipot_nuc_scores(ipot_t *pot, const void *logits, int logits_dtype, long long row_stride,
                     const int32_t *labels, int n_tokens, int vocab, float *aux_out, long long aux_stride,
                     int slot0);
+
+/*
+ * Context-reset rotary embedding (Sec. 3.4): the pot keeps its keys WITHOUT rotary embedding and every
+ * slot j carries position j, so positions run 0 .. len-1 again after each cycle.  With this mode on, the
+ * K rows passed to ipot_append_chunk are unrotated keys; the library maintains beside them a copy in
+ * which slot j is rotated at position j (ipot_view_rope): appended rows are rotated at the slots they
+ * land in, and a cycle rotates every row it moves at its new slot, inside the same kernels that move
+ * the rows, so no separate pass over the pot follows a cycle.  The CaP queries of
+ * ipot_score_and_compress attend to the rotated copy (the caller rotates Q_cap at the CaP's positions
+ * len .. len + cap_rows - 1); ipot_view keeps returning the unrotated keys.
+ *   cos_table, sin_table : device, [pot_size][d / 2] in the pot's dtype, 16-byte aligned, caller-owned
+ *                          and read by every later append and cycle until ipot_destroy: cos and sin of
+ *                          position x frequency (the paper fixes no base or scaling; they are the
+ *                          model's).
+ *   pairing              : IPOT_ROPE_HALF (channel c with c + d/2) or IPOT_ROPE_INTERLEAVED (2c, 2c + 1).
+ * The rotation is evaluated in single precision as lo' = fma(lo, cos, -(hi * sin)),
+ * hi' = fma(hi, cos, lo * sin) and rounded once to the pot's dtype.
+ * Allowed only while the pot is empty (len == 0; else IPOT_E_STATE); needs d * element size to be a
+ * multiple of 32 bytes (IPOT_E_INVALID otherwise).  The first call allocates the copy (pot_size rows per
+ * unit; synchronises the stream; IPOT_E_NOMEM).  The mode stays on for the life of the pot.
+ */
+int ipot_enable_rope(ipot_t *pot, const void *cos_table, const void *sin_table, int pairing);
+
+/* Borrowed device pointer to the rotated copy of the keys, [layers][batch][Hkv][pot_size][d]; rows >= len
+ * are undefined.  IPOT_E_STATE unless ipot_enable_rope was called. */
+int ipot_view_rope(ipot_t *pot, void **K_rot);
 
 /*
  * Borrowed device pointers to the pot ([layers][batch][Hkv][pot_size][d]) and

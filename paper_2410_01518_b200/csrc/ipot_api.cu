@@ -13,6 +13,7 @@
 #include "k_cap_self.cuh"
 #include "k_move.cuh"
 #include "k_novelty.cuh"
+#include "k_rope.cuh"
 #include "k_score_simt.cuh"
 #include "k_score_tc.cuh"
 #include "k_select.cuh"
@@ -26,10 +27,15 @@ struct ipot {
     int sm_count;
     int scorer;
     int G, units, elem_bytes, row_bytes;
-    int compact_slices;
+    int compact_slices, rope_slices;
     cudaStream_t stream;
     // device memory (library-owned)
     void *K, *V;
+    // CR-RoPE (ipot_enable_rope): K then holds the keys without rotary embedding, Krot the copy rotated at the slot
+    // numbers, which is what the scorers read; the tables are the caller's
+    void *Krot;
+    const void *rope_cos, *rope_sin;
+    int rope;            // 0 off, IPOT_ROPE_HALF, IPOT_ROPE_INTERLEAVED
     float *scores;       // [max_parts][units * pot_size]; array q holds [units][N] partial scores of the
                          // q-th block of 128 query rows (the SIMT scorer writes array 0 only)
     float *summed;       // [units][N]: sum of the partial arrays when there are several
@@ -74,6 +80,9 @@ constexpr size_t kNovCounterBytes = (size_t)(kNovMaxRows + 1) * sizeof(int);
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// the keys the CaP queries attend to
+const void *score_keys(const ipot *p) { return p->rope ? p->Krot : p->K; }
+
 int check_config(const ipot_config_t &c)
 {
     if (c.pot_size <= 0 || c.pot_size > 32768) return IPOT_E_INVALID;
@@ -89,7 +98,7 @@ int check_config(const ipot_config_t &c)
 void free_all(ipot *p)
 {
     tc_plan_destroy(p->tc);
-    cudaFree(p->K); cudaFree(p->V); cudaFree(p->scores); cudaFree(p->summed);
+    cudaFree(p->K); cudaFree(p->V); cudaFree(p->Krot); cudaFree(p->scores); cudaFree(p->summed);
     cudaFree(p->row_stats); cudaFree(p->cap_stats); cudaFree(p->nuc_mask); cudaFree(p->idx); cudaFree(p->status);
     cudaFree(p->stage_q); cudaFree(p->stage_kc); cudaFree(p->stage_aux); cudaFree(p->nov_scratch);
     if (p->ev) {
@@ -130,9 +139,9 @@ int launch_simt(ipot *p, const void *Q, const float2 *cap_stats, int M, int N)
     const float scale_log2e = (float)(1.4426950408889634 / std::sqrt((double)d));
     const size_t kstride = (size_t)p->cfg.pot_size * d;
     dim3 g1((M + kSimtRows - 1) / kSimtRows, p->units), g2((N + kSimtKeys - 1) / kSimtKeys, p->units);
-    cap_row_stats<T><<<g1, kSimtThreads, smem, p->stream>>>((const T *)Q, (const T *)p->K, p->row_stats, M, N, d, kstride, scale_log2e,
+    cap_row_stats<T><<<g1, kSimtThreads, smem, p->stream>>>((const T *)Q, (const T *)score_keys(p), p->row_stats, M, N, d, kstride, scale_log2e,
                                                             cap_stats, 0, 1);
-    cap_column_sums<T><<<g2, kSimtThreads, smem, p->stream>>>((const T *)Q, (const T *)p->K, p->row_stats, p->scores, M, N, d, kstride, scale_log2e);
+    cap_column_sums<T><<<g2, kSimtThreads, smem, p->stream>>>((const T *)Q, (const T *)score_keys(p), p->row_stats, p->scores, M, N, d, kstride, scale_log2e);
     p->launches += 2;
     IPOT_CUDA(cudaGetLastError());
     return IPOT_OK;
@@ -165,7 +174,7 @@ int run_scoring(ipot *p, const void *Q, const void *Kc, int cap_rows, const floa
     const float2 *cap_stats = Kc ? p->cap_stats : nullptr;
     if (scorer == IPOT_SCORER_TENSOR) {
         int n_launch = 0;
-        rc = tc_launch(p->tc, p->cfg, Q, p->K, cap_stats, p->scores, (size_t)p->units * p->cfg.pot_size, N, M, p->units, p->status,
+        rc = tc_launch(p->tc, p->cfg, Q, score_keys(p), cap_stats, p->scores, (size_t)p->units * p->cfg.pot_size, N, M, p->units, p->status,
                        p->stream, parts, &n_launch);
         p->launches += n_launch;
     } else {
@@ -188,6 +197,47 @@ int check_cycle_args(ipot *p, const void *Q, int cap_rows, const float *aux, boo
     return IPOT_OK;
 }
 
+template <typename T>
+void launch_compact_rope_t(ipot *p, dim3 grid, int keep, int N, int row_vecs, size_t unit_vecs)
+{
+    const int sv = row_vecs / 2 / p->rope_slices;
+    if (p->rope == IPOT_ROPE_INTERLEAVED)
+        compact_rope_kernel<T, true><<<grid, kMoveThreads, 0, p->stream>>>((uint4 *)p->K, (uint4 *)p->Krot, (const T *)p->rope_cos,
+                                                                          (const T *)p->rope_sin, p->idx, keep, N, row_vecs, sv, unit_vecs, p->status);
+    else
+        compact_rope_kernel<T, false><<<grid, kMoveThreads, 0, p->stream>>>((uint4 *)p->K, (uint4 *)p->Krot, (const T *)p->rope_cos,
+                                                                           (const T *)p->rope_sin, p->idx, keep, N, row_vecs, sv, unit_vecs, p->status);
+}
+
+void launch_compact_rope(ipot *p, dim3 grid, int keep, int N, int row_vecs, size_t unit_vecs)
+{
+    if (p->cfg.dtype == IPOT_F32) launch_compact_rope_t<float>(p, grid, keep, N, row_vecs, unit_vecs);
+    else launch_compact_rope_t<__nv_bfloat16>(p, grid, keep, N, row_vecs, unit_vecs);
+}
+
+// New key rows (src, unit stride src_unit_vecs) -> pot rows [len, len + n) unrotated and rotated.
+template <typename T>
+void launch_append_rope_t(ipot *p, const void *src, size_t src_unit_vecs, int n)
+{
+    const int row_vecs = p->row_bytes / 16;
+    const size_t items = (size_t)n * (row_vecs / 2), unit_vecs = (size_t)p->cfg.pot_size * row_vecs;
+    int pieces = (int)((items + (size_t)kMoveThreads * 4 - 1) / ((size_t)kMoveThreads * 4));
+    if (pieces < 1) pieces = 1;
+    dim3 grid(pieces, p->units);
+    if (p->rope == IPOT_ROPE_INTERLEAVED)
+        append_rope_kernel<T, true><<<grid, kMoveThreads, 0, p->stream>>>((const uint4 *)src, src_unit_vecs, (uint4 *)p->K, (uint4 *)p->Krot,
+                                                                         (const T *)p->rope_cos, (const T *)p->rope_sin, n, row_vecs, unit_vecs, p->len);
+    else
+        append_rope_kernel<T, false><<<grid, kMoveThreads, 0, p->stream>>>((const uint4 *)src, src_unit_vecs, (uint4 *)p->K, (uint4 *)p->Krot,
+                                                                          (const T *)p->rope_cos, (const T *)p->rope_sin, n, row_vecs, unit_vecs, p->len);
+}
+
+void launch_append_rope(ipot *p, const void *src, size_t src_unit_vecs, int n)
+{
+    if (p->cfg.dtype == IPOT_F32) launch_append_rope_t<float>(p, src, src_unit_vecs, n);
+    else launch_append_rope_t<__nv_bfloat16>(p, src, src_unit_vecs, n);
+}
+
 // Byte-column slices per row for the compaction grid: enough blocks to fill the device, slices of >= 64 bytes.
 int compact_slices(const ipot *p)
 {
@@ -195,6 +245,17 @@ int compact_slices(const ipot *p)
     int slices = 1;
     while (row_vecs % (slices * 2) == 0 && row_vecs / (slices * 2) >= 4 &&
            (long long)p->units * 2 * slices < 8LL * p->sm_count)
+        slices *= 2;
+    return slices;
+}
+
+// The same for the vector pairs (g, g + row_vecs / 2) of compact_rope_kernel: slices of >= 2 pairs.
+int rope_slices(const ipot *p)
+{
+    const int half_vecs = p->row_bytes / 32;
+    int slices = 1;
+    while (half_vecs % (slices * 2) == 0 && half_vecs / (slices * 2) >= 2 &&
+           (long long)p->units * slices < 8LL * p->sm_count)
         slices *= 2;
     return slices;
 }
@@ -216,10 +277,20 @@ int run_cycle(ipot *p, const void *Q, const void *Kc, int cap_rows, const float 
 
     const int row_vecs = p->row_bytes / 16;
     const int slices = p->compact_slices;
-    dim3 grid(slices, p->units, 2);
-    compact_kernel<<<grid, kMoveThreads, 0, p->stream>>>((uint4 *)p->K, (uint4 *)p->V, p->idx, keep, N, row_vecs,
-                                                        row_vecs / slices, (size_t)p->cfg.pot_size * row_vecs, p->status);
-    p->launches += 1;
+    const size_t unit_vecs = (size_t)p->cfg.pot_size * row_vecs;
+    if (!p->rope) {
+        dim3 grid(slices, p->units, 2);
+        compact_kernel<<<grid, kMoveThreads, 0, p->stream>>>((uint4 *)p->K, (uint4 *)p->V, p->idx, keep, N, row_vecs,
+                                                            row_vecs / slices, unit_vecs, p->status);
+        p->launches += 1;
+    } else {
+        // V as before (one tensor per launch); K through the kernel that also writes the rotated copy
+        dim3 gv(slices, p->units, 1), gk(p->rope_slices, p->units);
+        compact_kernel<<<gv, kMoveThreads, 0, p->stream>>>((uint4 *)p->V, (uint4 *)p->V, p->idx, keep, N, row_vecs,
+                                                          row_vecs / slices, unit_vecs, p->status);
+        launch_compact_rope(p, gk, keep, N, row_vecs, unit_vecs);
+        p->launches += 2;
+    }
     IPOT_CUDA(cudaGetLastError());
     if (ev) {
         IPOT_CUDA(cudaEventRecord(ev[4], p->stream));
@@ -323,6 +394,7 @@ int ipot_create_ex(const ipot_config_t *cfg, ipot_t **out)
         return IPOT_E_CUDA;
     }
     p->compact_slices = compact_slices(p);
+    p->rope_slices = rope_slices(p);
     tc_plan_init(p->tc, p->cfg, p->K, p->sm_count);
     *out = p;
     return IPOT_OK;
@@ -374,9 +446,18 @@ int ipot_append_chunk(ipot_t *p, const void *K, const void *V, int n)
     const size_t n_vecs = (size_t)n * row_vecs;
     int pieces = (int)((n_vecs + (size_t)kMoveThreads * kMoveVecs - 1) / ((size_t)kMoveThreads * kMoveVecs));
     if (pieces < 1) pieces = 1;
-    dim3 grid(pieces, p->units, 2);
-    append_kernel<<<grid, kMoveThreads, 0, p->stream>>>((const uint4 *)K, (const uint4 *)V, (uint4 *)p->K, (uint4 *)p->V,
-                                                       n_vecs, (size_t)p->cfg.pot_size * row_vecs, (size_t)p->len * row_vecs);
+    if (!p->rope) {
+        dim3 grid(pieces, p->units, 2);
+        append_kernel<<<grid, kMoveThreads, 0, p->stream>>>((const uint4 *)K, (const uint4 *)V, (uint4 *)p->K, (uint4 *)p->V,
+                                                           n_vecs, (size_t)p->cfg.pot_size * row_vecs, (size_t)p->len * row_vecs);
+    } else {
+        if (!p->rope_cos) return IPOT_E_STATE;
+        dim3 grid(pieces, p->units, 1);  // V as before; K through the kernel that also writes the rotated copy
+        append_kernel<<<grid, kMoveThreads, 0, p->stream>>>((const uint4 *)V, (const uint4 *)V, (uint4 *)p->V, (uint4 *)p->V,
+                                                           n_vecs, (size_t)p->cfg.pot_size * row_vecs, (size_t)p->len * row_vecs);
+        launch_append_rope(p, K, n_vecs, n);
+        p->launches += 1;
+    }
     p->launches += 1;
     IPOT_CUDA(cudaGetLastError());
     p->len += n;
@@ -391,6 +472,11 @@ int ipot_append_chunk_host(ipot_t *p, const void *K, const void *V, int n)
     char *dK = (char *)p->K + (size_t)p->len * p->row_bytes, *dV = (char *)p->V + (size_t)p->len * p->row_bytes;
     IPOT_CUDA(cudaMemcpy2DAsync(dK, dpitch, K, width, width, p->units, cudaMemcpyHostToDevice, p->stream));
     IPOT_CUDA(cudaMemcpy2DAsync(dV, dpitch, V, width, width, p->units, cudaMemcpyHostToDevice, p->stream));
+    if (p->rope) {  // the key rows are in place: rotate them into the copy
+        launch_append_rope(p, dK, (size_t)p->cfg.pot_size * (p->row_bytes / 16), n);
+        p->launches += 1;
+        IPOT_CUDA(cudaGetLastError());
+    }
     p->len += n;
     return IPOT_OK;
 }
@@ -502,6 +588,34 @@ int ipot_nuc_scores(ipot_t *p, const void *logits, int logits_dtype, long long r
     return logits_dtype == IPOT_F32
                ? launch_novelty<float>(p, logits, (size_t)row_stride, labels, n_tokens, vocab, aux_out, (size_t)aux_stride, slot0)
                : launch_novelty<__nv_bfloat16>(p, logits, (size_t)row_stride, labels, n_tokens, vocab, aux_out, (size_t)aux_stride, slot0);
+}
+
+int ipot_enable_rope(ipot_t *p, const void *cos_table, const void *sin_table, int pairing)
+{
+    if (!p || !cos_table || !sin_table || !aligned16(cos_table) || !aligned16(sin_table)) return IPOT_E_INVALID;
+    if (pairing != IPOT_ROPE_HALF && pairing != IPOT_ROPE_INTERLEAVED) return IPOT_E_INVALID;
+    if (p->row_bytes % 32) return IPOT_E_INVALID;  // a row must split into two halves of whole 16-byte vectors
+    if (p->len != 0) return IPOT_E_STATE;
+    if (!p->Krot) {
+        IPOT_CUDA(cudaStreamSynchronize(p->stream));
+        if (cudaMalloc(&p->Krot, (size_t)p->units * p->cfg.pot_size * p->row_bytes) != cudaSuccess) {
+            cudaGetLastError();
+            p->Krot = nullptr;
+            return IPOT_E_NOMEM;
+        }
+    }
+    p->rope_cos = cos_table;
+    p->rope_sin = sin_table;
+    p->rope = pairing;
+    return IPOT_OK;
+}
+
+int ipot_view_rope(ipot_t *p, void **K_rot)
+{
+    if (!p || !K_rot) return IPOT_E_INVALID;
+    if (!p->rope) return IPOT_E_STATE;
+    *K_rot = p->Krot;
+    return IPOT_OK;
 }
 
 int ipot_view(ipot_t *p, void **K, void **V, int *len)

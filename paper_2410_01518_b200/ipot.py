@@ -20,6 +20,7 @@ IPOT_OK, IPOT_E_INVALID, IPOT_E_STATE, IPOT_E_NOMEM, IPOT_E_CUDA, IPOT_E_TIMEOUT
 IPOT_NOALLOC_MAX_ROWS = 65536
 IPOT_BF16, IPOT_F32 = 0, 1
 IPOT_SCORER_AUTO, IPOT_SCORER_SIMT, IPOT_SCORER_TENSOR = 0, 1, 2
+IPOT_ROPE_HALF, IPOT_ROPE_INTERLEAVED = 1, 2
 
 # every symbol include/ipot.h declares
 SYMBOLS = [
@@ -29,7 +30,7 @@ SYMBOLS = [
     "ipot_last_indices", "ipot_last_scores", "ipot_sync_status", "ipot_set_profiling",
     "ipot_kernel_ms", "ipot_launch_count", "ipot_strerror", "ipot_cap_scores_noalloc",
     "ipot_score_and_compress_cap", "ipot_score_only_cap", "ipot_score_and_compress_cap_host",
-    "ipot_nuc_scores",
+    "ipot_nuc_scores", "ipot_enable_rope", "ipot_view_rope",
 ]
 
 
@@ -77,6 +78,8 @@ def lib() -> C.CDLL:
         L.ipot_score_only_cap.argtypes = [vp, vp, vp, ip, vp]
         L.ipot_score_and_compress_cap_host.argtypes = [vp, vp, vp, ip, vp, vp]
         L.ipot_nuc_scores.argtypes = [vp, vp, ip, C.c_longlong, vp, ip, ip, vp, C.c_longlong, ip]
+        L.ipot_enable_rope.argtypes = [vp, vp, vp, ip]
+        L.ipot_view_rope.argtypes = [vp, C.POINTER(vp)]
         L.ipot_view.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(ip)]
         L.ipot_last_indices.argtypes = [vp, C.POINTER(vp)]
         L.ipot_last_scores.argtypes = [vp, C.POINTER(vp), C.POINTER(ip)]
@@ -186,6 +189,17 @@ def ipot_score_only_cap(h, Q_cap, K_cap, cap_rows, aux_scores=None) -> None:
 def ipot_nuc_scores(h, logits, logits_dtype, row_stride, labels, n_tokens, vocab, aux_out, aux_stride, slot0) -> None:
     _check(lib().ipot_nuc_scores(h, _ptr(logits), logits_dtype, row_stride, _ptr(labels), n_tokens, vocab,
                                  _ptr(aux_out), aux_stride, slot0), "ipot_nuc_scores")
+
+
+def ipot_enable_rope(h, cos_table, sin_table, pairing) -> None:
+    _check(lib().ipot_enable_rope(h, _ptr(cos_table), _ptr(sin_table), pairing), "ipot_enable_rope")
+
+
+def ipot_view_rope(h) -> int:
+    """-> device address of the rotated copy of the keys."""
+    p = C.c_void_p()
+    _check(lib().ipot_view_rope(h, C.byref(p)), "ipot_view_rope")
+    return p.value
 
 
 def ipot_view(h):

@@ -57,12 +57,24 @@ def read_results(h, cfg: inputs.CcdConfig, n_before: int):
     return u, idx, K, V
 
 
+def read_rotated(h, cfg: inputs.CcdConfig, rows: int) -> np.ndarray:
+    """The first `rows` rows of the rotated copy of the keys, [units][rows][d] storage bits."""
+    assert ipot.ipot_sync_status(h) == 0
+    shape = (cfg.units, cfg.pot_size, cfg.d)
+    return from_dev_bits(ipot.device_array(ipot.ipot_view_rope(h), shape, cfg.dtype)[:, :rows], cfg.dtype)
+
+
 def gpu_cycle(cfg: inputs.CcdConfig, t: dict, scorer=ipot.IPOT_SCORER_AUTO, n=None):
     """Fill a fresh pot with t['K'], t['V'] (first n rows), run one cycle, read everything back."""
     n = cfg.pot_size if n is None else n
     h = make_pot(cfg, max_cap_rows=t["Q"].shape[3])
+    keep_alive = []
     try:
         ipot.ipot_set_scorer(h, scorer)
+        if t.get("rope") is not None:  # Sec. 3.4: t["K"] holds unrotated keys, the library keeps the rotated copy
+            cos_t, sin_t, inter = t["rope"]
+            keep_alive = [to_dev(cos_t, cfg.dtype), to_dev(sin_t, cfg.dtype)]
+            ipot.ipot_enable_rope(h, keep_alive[0], keep_alive[1], ipot.IPOT_ROPE_INTERLEAVED if inter else ipot.IPOT_ROPE_HALF)
         Kd, Vd = to_dev(t["K"][:, :, :, :n], cfg.dtype), to_dev(t["V"][:, :, :, :n], cfg.dtype)
         Qd = to_dev(t["Q"], cfg.dtype)
         auxd = torch.from_numpy(np.ascontiguousarray(t["aux"][:, :n])).cuda()
@@ -72,7 +84,10 @@ def gpu_cycle(cfg: inputs.CcdConfig, t: dict, scorer=ipot.IPOT_SCORER_AUTO, n=No
                                              auxd if cfg.nuc_slots > 0 else None)
         else:
             ipot.ipot_score_and_compress(h, Qd, t["Q"].shape[3], auxd if cfg.nuc_slots > 0 else None)
-        return read_results(h, cfg, n)
+        res = read_results(h, cfg, n)
+        if t.get("rope") is not None:
+            res = res + (read_rotated(h, cfg, cfg.keep),)
+        return res
     finally:
         ipot.ipot_destroy(h)
 
@@ -105,14 +120,21 @@ def compare_cycle(cfg, t, gpu, units=None, n=None):
     Returns (units whose index list is identical to the checker's, units compared)."""
     n = cfg.pot_size if n is None else n
     K_in, V_in = t["K"][:, :, :, :n], t["V"][:, :, :, :n]
-    ref = oracle.cycle(t["Q"], K_in, V_in, t["aux"][:, :n], cfg.keep, cfg.nuc_slots, units=units, K_cap=t.get("K_cap"))
-    u, idx, K, V = gpu
+    ref = oracle.cycle(t["Q"], K_in, V_in, t["aux"][:, :n], cfg.keep, cfg.nuc_slots, units=units, K_cap=t.get("K_cap"),
+                       rope=t.get("rope"))
+    u, idx, K, V = gpu[:4]
     Kf, Vf = K_in.reshape(cfg.units, n, cfg.d), V_in.reshape(cfg.units, n, cfg.d)
     M = cfg.G * t["Q"].shape[3]
     nuc = [oracle.nuc_top(t["aux"][b, :n], cfg.nuc_slots) for b in range(cfg.batch)]
     identical = 0
     for k, unit in enumerate(ref["units"]):
         b = (unit // cfg.Hkv) % cfg.batch
-        identical += check_unit(cfg, u[unit], idx[unit], K[unit], V[unit], Kf[unit], Vf[unit],
-                                ref["u"][k], ref["idx"][k], nuc[b], M, ref["K"][k], ref["V"][k])
+        same = check_unit(cfg, u[unit], idx[unit], K[unit], V[unit], Kf[unit], Vf[unit],
+                          ref["u"][k], ref["idx"][k], nuc[b], M, ref["K"][k], ref["V"][k])
+        identical += same
+        if t.get("rope") is not None:  # the rotated copy: the survivors rotated at their new slot numbers, bit for bit
+            cos_t, sin_t, inter = t["rope"]
+            assert (gpu[4][unit] == oracle.rope_rows(Kf[unit][idx[unit]], np.arange(cfg.keep), cos_t, sin_t, inter)).all()
+            if same:
+                assert (gpu[4][unit] == ref["K_rot"][k]).all()
     return identical, len(ref["units"])
