@@ -112,7 +112,7 @@ class ClockSampler:
         return out
 
 
-def cpu_baseline(cfg, ring, K0, V0, n_units_sample, threads=None):
+def cpu_baseline(cfg, ring, K0, V0, n_units_sample, threads=None, rope=False):
     """The checker, as it stands, on a sample of the units of one cycle."""
     import oracle
     if threads:
@@ -121,9 +121,10 @@ def cpu_baseline(cfg, ring, K0, V0, n_units_sample, threads=None):
     K = np.concatenate([K0, t["K"]], axis=3)
     V = np.concatenate([V0, t["V"]], axis=3)
     units = np.linspace(0, cfg.units - 1, n_units_sample).astype(np.int32)
-    oracle.cycle(t["Q"], K, V, t["aux"], cfg.keep, cfg.nuc_slots, units=units[:1], K_cap=t.get("K_cap"))  # load the library
+    rope = inputs.make_rope_table(cfg.pot_size, cfg.d, cfg.dtype) + (False,) if rope else None
+    oracle.cycle(t["Q"], K, V, t["aux"], cfg.keep, cfg.nuc_slots, units=units[:1], K_cap=t.get("K_cap"), rope=rope)  # load the library
     t0 = time.perf_counter()
-    oracle.cycle(t["Q"], K, V, t["aux"], cfg.keep, cfg.nuc_slots, units=units, K_cap=t.get("K_cap"))
+    oracle.cycle(t["Q"], K, V, t["aux"], cfg.keep, cfg.nuc_slots, units=units, K_cap=t.get("K_cap"), rope=rope)
     dt = time.perf_counter() - t0
     cycles_per_s = (len(units) / cfg.units) / dt
     return cycles_per_s, dt, len(units), oracle.max_threads()
@@ -151,10 +152,10 @@ def run_reference(args, cfg):
     ring, K0, V0 = gen_ring(small, n_new, args.cap_keys)
     n_sample = min(small.units, 16)
     for _ in range(args.warmup):
-        cpu_baseline(small, ring, K0, V0, 1)
+        cpu_baseline(small, ring, K0, V0, 1, rope=args.rope)
     times = []
     for _ in range(args.steps):
-        _, dt, n_units, threads = cpu_baseline(small, ring, K0, V0, n_sample)
+        _, dt, n_units, threads = cpu_baseline(small, ring, K0, V0, n_sample, rope=args.rope)
         times.append(dt)
     ms = float(np.mean(times)) * 1e3 * cfg.units / n_sample  # one full cycle, extrapolated
     value = 1e3 / ms
@@ -162,7 +163,7 @@ def run_reference(args, cfg):
         "impl": "reference", "metric": "ccd_cycles_per_s", "value": value, "unit": "cycles/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": config_dict(cfg, n_new, N, args.cap_keys),
+        "config": config_dict(cfg, n_new, N, args.cap_keys, getattr(args, "rope", False)),
         "cpu_baseline": {"value": value, "unit": "cycles/s", "cores": threads, "kind": "oracle",
                          "sample": f"{n_sample} of {cfg.units} units of one cycle per step (units are independent and "
                                    f"equal-sized); full-cycle time extrapolated"},
@@ -290,10 +291,10 @@ def run_novelty(args):
         dist.destroy_process_group()
 
 
-def config_dict(cfg, n_new, N, cap_keys=False):
+def config_dict(cfg, n_new, N, cap_keys=False, rope=False):
     return {"workload": f"configs[{cfg.cfg_id - 1}] {cfg.name}: one CCD cycle per step "
                         f"(append {n_new} rows, distil {N} -> {cfg.keep})"
-                        + ("; CaP keys inside the softmax" if cap_keys else ""),
+                        + ("; CaP keys inside the softmax" if cap_keys else "") + ("; rotary mode" if rope else ""),
             "layers": cfg.layers, "batch": cfg.batch, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "d": cfg.d,
             "pot_size": cfg.pot_size, "keep": cfg.keep, "nuc_slots": cfg.nuc_slots, "cap_rows": cfg.cap_rows,
             "units": cfg.units, "l2": "inputs_larger_than_l2" if cfg.units * N * cfg.d * cfg.elem_bytes * 2 > 126e6
@@ -311,6 +312,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cap-keys", action="store_true",
                     help="score with the CaP's own keys inside the softmax (the Appendix B listing read literally)")
+    ap.add_argument("--rope", action="store_true",
+                    help="context-reset rotary mode: unrotated keys in the pot, the row movers keep a rotated copy")
     ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (profiling small cases)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -357,6 +360,9 @@ def main():
                             dtype=ipot.IPOT_BF16 if cfg.dtype == "bf16" else ipot.IPOT_F32,
                             nuc_slots=cfg.nuc_slots, max_cap_rows=cfg.cap_rows)
     ipot.ipot_set_scorer(h, {"auto": 0, "simt": 1, "tensor": 2}[args.scorer])
+    if args.rope:
+        rope_tables = [dev(a) for a in inputs.make_rope_table(cfg.pot_size, cfg.d, cfg.dtype)]
+        ipot.ipot_enable_rope(h, rope_tables[0], rope_tables[1], ipot.IPOT_ROPE_HALF)
     stream = torch.cuda.current_stream()
     ipot.ipot_set_stream(h, stream.cuda_stream)
     ipot.ipot_append_chunk(h, K0d, V0d, cfg.keep)
@@ -428,7 +434,8 @@ def main():
     units, e, d, M = cfg.units, cfg.elem_bytes, cfg.d, cfg.G * cfg.cap_rows
     score_bytes = units * (N * d * e + M * d * e + 4 * N)      # K once + Q + scores out
     score_flops = 2.0 * units * M * N * d
-    compact_bytes = units * 4 * cfg.keep * d * e                # K and V, read + write, all kept rows
+    # K and V, read + write, all kept rows; in rotary mode the rotated copy of K is written as well
+    compact_bytes = units * (5 if args.rope else 4) * cfg.keep * d * e
     names = ["nuc_rank", "cap_score", "select", "compact"]
     # the dominant kernel; scoring and compaction are close, scoring is named unless compaction is clearly longer
     dom = 3 if kms[3] > 1.05 * kms[1] else 1
@@ -453,7 +460,7 @@ def main():
         "metric": "ccd_cycles_per_s", "value": value, "unit": "cycles/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
-        "config": config_dict(cfg, n_new, N, args.cap_keys),
+        "config": config_dict(cfg, n_new, N, args.cap_keys, getattr(args, "rope", False)),
         "pot_tokens_per_s": value * N * cfg.batch,
         "layer_cycles_per_s": value * cfg.layers,
         "clocks": clocks,
@@ -464,7 +471,7 @@ def main():
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         n_sample = min(cfg.units, 256)
-        v, dt, n_units, threads = cpu_baseline(cfg, ring, K0, V0, n_sample)
+        v, dt, n_units, threads = cpu_baseline(cfg, ring, K0, V0, n_sample, rope=args.rope)
         line["cpu_baseline"] = {"value": v, "unit": "cycles/s", "cores": threads, "kind": "oracle",
                                 "sample": f"{n_units} of {cfg.units} units of one cycle in {dt:.1f} s; "
                                           f"full-cycle rate extrapolated (units are independent and equal-sized)"}

@@ -197,45 +197,43 @@ int check_cycle_args(ipot *p, const void *Q, int cap_rows, const float *aux, boo
     return IPOT_OK;
 }
 
+// One launch: z = 0 gathers the unrotated keys and writes the rotated copy, z = 1 gathers the values.
 template <typename T>
-void launch_compact_rope_t(ipot *p, dim3 grid, int keep, int N, int row_vecs, size_t unit_vecs)
+void launch_compact_rope_t(ipot *p, int keep, int N, int row_vecs, size_t unit_vecs)
 {
-    const int sv = row_vecs / 2 / p->rope_slices;
-    if (p->rope == IPOT_ROPE_INTERLEAVED)
-        compact_rope_kernel<T, true><<<grid, kMoveThreads, 0, p->stream>>>((uint4 *)p->K, (uint4 *)p->Krot, (const T *)p->rope_cos,
-                                                                          (const T *)p->rope_sin, p->idx, keep, N, row_vecs, sv, unit_vecs, p->status);
-    else
-        compact_rope_kernel<T, false><<<grid, kMoveThreads, 0, p->stream>>>((uint4 *)p->K, (uint4 *)p->Krot, (const T *)p->rope_cos,
-                                                                           (const T *)p->rope_sin, p->idx, keep, N, row_vecs, sv, unit_vecs, p->status);
+    const int ks = p->rope_slices, vs = p->compact_slices;
+    dim3 grid(ks > vs ? ks : vs, p->units, 2);
+    auto kern = p->rope == IPOT_ROPE_INTERLEAVED ? compact_rope_kernel<T, true> : compact_rope_kernel<T, false>;
+    kern<<<grid, kMoveThreads, 0, p->stream>>>((uint4 *)p->K, (uint4 *)p->Krot, (const T *)p->rope_cos, (const T *)p->rope_sin, p->idx,
+                                               keep, N, row_vecs, ks, row_vecs / 2 / ks, unit_vecs, p->status, (uint4 *)p->V, vs,
+                                               row_vecs / vs);
 }
 
-void launch_compact_rope(ipot *p, dim3 grid, int keep, int N, int row_vecs, size_t unit_vecs)
+void launch_compact_rope(ipot *p, int keep, int N, int row_vecs, size_t unit_vecs)
 {
-    if (p->cfg.dtype == IPOT_F32) launch_compact_rope_t<float>(p, grid, keep, N, row_vecs, unit_vecs);
-    else launch_compact_rope_t<__nv_bfloat16>(p, grid, keep, N, row_vecs, unit_vecs);
+    if (p->cfg.dtype == IPOT_F32) launch_compact_rope_t<float>(p, keep, N, row_vecs, unit_vecs);
+    else launch_compact_rope_t<__nv_bfloat16>(p, keep, N, row_vecs, unit_vecs);
 }
 
-// New key rows (src, unit stride src_unit_vecs) -> pot rows [len, len + n) unrotated and rotated.
+// New key rows (src, unit stride src_unit_vecs) -> pot rows [len, len + n) unrotated and rotated; if srcV is not
+// NULL the same launch copies the value rows ([units][n rows]) into the pot.
 template <typename T>
-void launch_append_rope_t(ipot *p, const void *src, size_t src_unit_vecs, int n)
+void launch_append_rope_t(ipot *p, const void *src, size_t src_unit_vecs, const void *srcV, int n)
 {
     const int row_vecs = p->row_bytes / 16;
     const size_t items = (size_t)n * (row_vecs / 2), unit_vecs = (size_t)p->cfg.pot_size * row_vecs;
     int pieces = (int)((items + (size_t)kMoveThreads * 4 - 1) / ((size_t)kMoveThreads * 4));
     if (pieces < 1) pieces = 1;
-    dim3 grid(pieces, p->units);
-    if (p->rope == IPOT_ROPE_INTERLEAVED)
-        append_rope_kernel<T, true><<<grid, kMoveThreads, 0, p->stream>>>((const uint4 *)src, src_unit_vecs, (uint4 *)p->K, (uint4 *)p->Krot,
-                                                                         (const T *)p->rope_cos, (const T *)p->rope_sin, n, row_vecs, unit_vecs, p->len);
-    else
-        append_rope_kernel<T, false><<<grid, kMoveThreads, 0, p->stream>>>((const uint4 *)src, src_unit_vecs, (uint4 *)p->K, (uint4 *)p->Krot,
-                                                                          (const T *)p->rope_cos, (const T *)p->rope_sin, n, row_vecs, unit_vecs, p->len);
+    dim3 grid(pieces, p->units, srcV ? 2 : 1);
+    auto kern = p->rope == IPOT_ROPE_INTERLEAVED ? append_rope_kernel<T, true> : append_rope_kernel<T, false>;
+    kern<<<grid, kMoveThreads, 0, p->stream>>>((const uint4 *)src, src_unit_vecs, (uint4 *)p->K, (uint4 *)p->Krot, (const T *)p->rope_cos,
+                                               (const T *)p->rope_sin, n, row_vecs, unit_vecs, p->len, (const uint4 *)srcV, (uint4 *)p->V);
 }
 
-void launch_append_rope(ipot *p, const void *src, size_t src_unit_vecs, int n)
+void launch_append_rope(ipot *p, const void *src, size_t src_unit_vecs, const void *srcV, int n)
 {
-    if (p->cfg.dtype == IPOT_F32) launch_append_rope_t<float>(p, src, src_unit_vecs, n);
-    else launch_append_rope_t<__nv_bfloat16>(p, src, src_unit_vecs, n);
+    if (p->cfg.dtype == IPOT_F32) launch_append_rope_t<float>(p, src, src_unit_vecs, srcV, n);
+    else launch_append_rope_t<__nv_bfloat16>(p, src, src_unit_vecs, srcV, n);
 }
 
 // Byte-column slices per row for the compaction grid: enough blocks to fill the device, slices of >= 64 bytes.
@@ -284,12 +282,8 @@ int run_cycle(ipot *p, const void *Q, const void *Kc, int cap_rows, const float 
                                                             row_vecs / slices, unit_vecs, p->status);
         p->launches += 1;
     } else {
-        // V as before (one tensor per launch); K through the kernel that also writes the rotated copy
-        dim3 gv(slices, p->units, 1), gk(p->rope_slices, p->units);
-        compact_kernel<<<gv, kMoveThreads, 0, p->stream>>>((uint4 *)p->V, (uint4 *)p->V, p->idx, keep, N, row_vecs,
-                                                          row_vecs / slices, unit_vecs, p->status);
-        launch_compact_rope(p, gk, keep, N, row_vecs, unit_vecs);
-        p->launches += 2;
+        launch_compact_rope(p, keep, N, row_vecs, unit_vecs);
+        p->launches += 1;
     }
     IPOT_CUDA(cudaGetLastError());
     if (ev) {
@@ -451,12 +445,7 @@ int ipot_append_chunk(ipot_t *p, const void *K, const void *V, int n)
         append_kernel<<<grid, kMoveThreads, 0, p->stream>>>((const uint4 *)K, (const uint4 *)V, (uint4 *)p->K, (uint4 *)p->V,
                                                            n_vecs, (size_t)p->cfg.pot_size * row_vecs, (size_t)p->len * row_vecs);
     } else {
-        if (!p->rope_cos) return IPOT_E_STATE;
-        dim3 grid(pieces, p->units, 1);  // V as before; K through the kernel that also writes the rotated copy
-        append_kernel<<<grid, kMoveThreads, 0, p->stream>>>((const uint4 *)V, (const uint4 *)V, (uint4 *)p->V, (uint4 *)p->V,
-                                                           n_vecs, (size_t)p->cfg.pot_size * row_vecs, (size_t)p->len * row_vecs);
-        launch_append_rope(p, K, n_vecs, n);
-        p->launches += 1;
+        launch_append_rope(p, K, n_vecs, V, n);
     }
     p->launches += 1;
     IPOT_CUDA(cudaGetLastError());
@@ -473,7 +462,7 @@ int ipot_append_chunk_host(ipot_t *p, const void *K, const void *V, int n)
     IPOT_CUDA(cudaMemcpy2DAsync(dK, dpitch, K, width, width, p->units, cudaMemcpyHostToDevice, p->stream));
     IPOT_CUDA(cudaMemcpy2DAsync(dV, dpitch, V, width, width, p->units, cudaMemcpyHostToDevice, p->stream));
     if (p->rope) {  // the key rows are in place: rotate them into the copy
-        launch_append_rope(p, dK, (size_t)p->cfg.pot_size * (p->row_bytes / 16), n);
+        launch_append_rope(p, dK, (size_t)p->cfg.pot_size * (p->row_bytes / 16), nullptr, n);
         p->launches += 1;
         IPOT_CUDA(cudaGetLastError());
     }

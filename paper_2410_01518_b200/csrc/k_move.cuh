@@ -11,15 +11,11 @@ namespace ipotk {
 constexpr int kMoveThreads = 256;
 constexpr int kMoveVecs = 8;  // 16-byte vectors in flight per thread
 
-// grid (pieces, units, 2): tensor z of unit y; src is [units][n_vecs], dst is the pot.
-__global__ void __launch_bounds__(kMoveThreads)
-append_kernel(const uint4 *__restrict__ srcK, const uint4 *__restrict__ srcV, uint4 *__restrict__ potK,
-              uint4 *__restrict__ potV, size_t n_vecs, size_t unit_vecs, size_t first_vec)
+// One block's share of a copy of n_vecs vectors: pieces blocks of kMoveThreads threads, block `piece`.
+__device__ __forceinline__ void append_body(const uint4 *__restrict__ src, uint4 *__restrict__ dst, size_t n_vecs, int piece, int pieces)
 {
-    const uint4 *src = (blockIdx.z ? srcV : srcK) + (size_t)blockIdx.y * n_vecs;
-    uint4 *dst = (blockIdx.z ? potV : potK) + (size_t)blockIdx.y * unit_vecs + first_vec;
-    const size_t stride = (size_t)gridDim.x * kMoveThreads;
-    size_t v = (size_t)blockIdx.x * kMoveThreads + threadIdx.x;
+    const size_t stride = (size_t)pieces * kMoveThreads;
+    size_t v = (size_t)piece * kMoveThreads + threadIdx.x;
     for (; v + (kMoveVecs - 1) * stride < n_vecs; v += kMoveVecs * stride) {
         uint4 t[kMoveVecs];
 #pragma unroll
@@ -30,6 +26,16 @@ append_kernel(const uint4 *__restrict__ srcK, const uint4 *__restrict__ srcV, ui
     for (; v < n_vecs; v += stride) dst[v] = __ldg(src + v);
 }
 
+// grid (pieces, units, 2): tensor z of unit y; src is [units][n_vecs], dst is the pot.
+__global__ void __launch_bounds__(kMoveThreads)
+append_kernel(const uint4 *__restrict__ srcK, const uint4 *__restrict__ srcV, uint4 *__restrict__ potK,
+              uint4 *__restrict__ potV, size_t n_vecs, size_t unit_vecs, size_t first_vec)
+{
+    const uint4 *src = (blockIdx.z ? srcV : srcK) + (size_t)blockIdx.y * n_vecs;
+    uint4 *dst = (blockIdx.z ? potV : potK) + (size_t)blockIdx.y * unit_vecs + first_vec;
+    append_body(src, dst, n_vecs, blockIdx.x, gridDim.x);
+}
+
 // In-place gather.  grid (slices, units, 2).  A block owns byte columns
 // [slice * slice_vecs, (slice + 1) * slice_vecs) (in 16-byte vectors) of every
 // row of one tensor of one unit, so blocks never touch the same bytes.  idx is
@@ -38,12 +44,10 @@ append_kernel(const uint4 *__restrict__ srcK, const uint4 *__restrict__ srcV, ui
 // writes land in rows below the next chunk's first row, and every later source
 // row lies at or above it, so nothing that is still needed is overwritten.
 // Rows with idx[r] == r are left alone.
-__global__ void __launch_bounds__(kMoveThreads)
-compact_kernel(uint4 *__restrict__ potK, uint4 *__restrict__ potV, const int32_t *__restrict__ idx,
-               int keep, int N, int row_vecs, int slice_vecs, size_t unit_vecs, int *status)
+// base: the block's first vector of row 0 (its byte-column slice of one tensor of one unit)
+__device__ __forceinline__ void compact_body(uint4 *__restrict__ base, const int32_t *__restrict__ ix, int keep, int N,
+                                             int row_vecs, int slice_vecs, int *status)
 {
-    uint4 *base = (blockIdx.z ? potV : potK) + (size_t)blockIdx.y * unit_vecs + (size_t)blockIdx.x * slice_vecs;
-    const int32_t *ix = idx + (size_t)blockIdx.y * keep;
     const int rows_per_pass = kMoveThreads / slice_vecs;  // rows covered by one vector per thread
     const int chunk_rows = rows_per_pass * kMoveVecs;
     const int my_row = threadIdx.x / slice_vecs, my_vec = threadIdx.x - my_row * slice_vecs;
@@ -70,6 +74,14 @@ compact_kernel(uint4 *__restrict__ potK, uint4 *__restrict__ potV, const int32_t
             if (src[i] >= 0) base[(size_t)r * row_vecs + my_vec] = t[i];
         }
     }
+}
+
+__global__ void __launch_bounds__(kMoveThreads)
+compact_kernel(uint4 *__restrict__ potK, uint4 *__restrict__ potV, const int32_t *__restrict__ idx,
+               int keep, int N, int row_vecs, int slice_vecs, size_t unit_vecs, int *status)
+{
+    uint4 *base = (blockIdx.z ? potV : potK) + (size_t)blockIdx.y * unit_vecs + (size_t)blockIdx.x * slice_vecs;
+    compact_body(base, idx + (size_t)blockIdx.y * keep, keep, N, row_vecs, slice_vecs, status);
 }
 
 }  // namespace ipotk

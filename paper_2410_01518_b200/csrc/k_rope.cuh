@@ -64,34 +64,53 @@ __device__ __forceinline__ void rope_pair(float lo, float hi, float cs, float sn
     hi_out = __fmaf_rn(hi, cs, __fmul_rn(lo, sn));
 }
 
-// Rotates vectors g (a) and g + half_vecs (b) of a row at position pos.  cos_t, sin_t: [positions][d / 2].
+// The table vectors a thread needs for vectors g and g + half_vecs of a row at position pos (cos_t, sin_t:
+// [positions][d / 2]): half pairing - cos and sin of frequencies g * VE .. (2 vectors); interleaved - a vector
+// holds VE / 2 pairs, so each of the two data vectors needs half a table vector, fetched as the 16-byte vector
+// that contains it (4 vectors: cos a, sin a, cos b, sin b).
+template <typename T, bool kInterleaved> struct RopeTab {
+    uint4 v[kInterleaved ? 4 : 2];
+    __device__ __forceinline__ void load(int g, int half_vecs, int pos, const T *__restrict__ cos_t, const T *__restrict__ sin_t)
+    {
+        constexpr int VE = RopeVec<T>::kElems;
+        const size_t trow = (size_t)pos * half_vecs * VE;  // d / 2 = half_vecs * VE table entries per position
+        if (!kInterleaved) {
+            v[0] = __ldg(reinterpret_cast<const uint4 *>(cos_t + trow + (size_t)g * VE));
+            v[1] = __ldg(reinterpret_cast<const uint4 *>(sin_t + trow + (size_t)g * VE));
+        } else {
+            const int fa = g * (VE / 2), fb = (g + half_vecs) * (VE / 2);
+            v[0] = __ldg(reinterpret_cast<const uint4 *>(cos_t + trow + (fa / VE) * VE));
+            v[1] = __ldg(reinterpret_cast<const uint4 *>(sin_t + trow + (fa / VE) * VE));
+            v[2] = __ldg(reinterpret_cast<const uint4 *>(cos_t + trow + (fb / VE) * VE));
+            v[3] = __ldg(reinterpret_cast<const uint4 *>(sin_t + trow + (fb / VE) * VE));
+        }
+    }
+};
+
+// Rotates vectors g (a) and g + half_vecs (b) of a row with the table vectors loaded for its position.
 template <typename T, bool kInterleaved>
-__device__ __forceinline__ void rope_two_vectors(const uint4 &a, const uint4 &b, int g, int half_vecs, int pos,
-                                                 const T *__restrict__ cos_t, const T *__restrict__ sin_t,
-                                                 uint4 &a_out, uint4 &b_out)
+__device__ __forceinline__ void rope_apply(const uint4 &a, const uint4 &b, int g, int half_vecs, const RopeTab<T, kInterleaved> &tab,
+                                           uint4 &a_out, uint4 &b_out)
 {
     constexpr int VE = RopeVec<T>::kElems;
-    const size_t trow = (size_t)pos * half_vecs * VE;  // d / 2 = half_vecs * VE table entries per position
     float xa[VE], xb[VE], ya[VE], yb[VE];
     RopeVec<T>::unpack(a, xa);
     RopeVec<T>::unpack(b, xb);
     if (!kInterleaved) {
         // a holds channels g * VE .. (the "lo" halves), b their partners c + d/2; frequencies g * VE ..
         float cs[VE], sn[VE];
-        RopeVec<T>::unpack(__ldg(reinterpret_cast<const uint4 *>(cos_t + trow + (size_t)g * VE)), cs);
-        RopeVec<T>::unpack(__ldg(reinterpret_cast<const uint4 *>(sin_t + trow + (size_t)g * VE)), sn);
+        RopeVec<T>::unpack(tab.v[0], cs);
+        RopeVec<T>::unpack(tab.v[1], sn);
 #pragma unroll
         for (int i = 0; i < VE; ++i) rope_pair(xa[i], xb[i], cs[i], sn[i], ya[i], yb[i]);
     } else {
-        // vector v holds the pairs (2c, 2c + 1) with c = v * VE / 2 ..: VE / 2 frequencies per vector; the table
-        // entries of a and of b are each half a vector, fetched as the 16-byte vector that contains them
+        // vector v holds the pairs (2c, 2c + 1) with c = v * VE / 2 ..
         float csa[VE], sna[VE], csb[VE], snb[VE];
-        const int fa = g * (VE / 2), fb = (g + half_vecs) * (VE / 2);
-        RopeVec<T>::unpack(__ldg(reinterpret_cast<const uint4 *>(cos_t + trow + (fa / VE) * VE)), csa);
-        RopeVec<T>::unpack(__ldg(reinterpret_cast<const uint4 *>(sin_t + trow + (fa / VE) * VE)), sna);
-        RopeVec<T>::unpack(__ldg(reinterpret_cast<const uint4 *>(cos_t + trow + (fb / VE) * VE)), csb);
-        RopeVec<T>::unpack(__ldg(reinterpret_cast<const uint4 *>(sin_t + trow + (fb / VE) * VE)), snb);
-        const int oa = fa % VE, ob = fb % VE;  // 0 or VE / 2
+        RopeVec<T>::unpack(tab.v[0], csa);
+        RopeVec<T>::unpack(tab.v[1], sna);
+        RopeVec<T>::unpack(tab.v[kInterleaved ? 2 : 0], csb);
+        RopeVec<T>::unpack(tab.v[kInterleaved ? 3 : 1], snb);
+        const int oa = (g * (VE / 2)) % VE, ob = ((g + half_vecs) * (VE / 2)) % VE;  // 0 or VE / 2
 #pragma unroll
         for (int i = 0; i < VE / 2; ++i) {
             rope_pair(xa[2 * i], xa[2 * i + 1], oa ? csa[VE / 2 + i] : csa[i], oa ? sna[VE / 2 + i] : sna[i], ya[2 * i], ya[2 * i + 1]);
@@ -102,20 +121,63 @@ __device__ __forceinline__ void rope_two_vectors(const uint4 &a, const uint4 &b,
     b_out = RopeVec<T>::pack(yb);
 }
 
-// grid (pieces, units).  src: key rows of unit y at src + y * src_unit_vecs, n rows of row_vecs vectors; the rows
-// go to pot rows first_row ... of potK (unchanged) and potKrot (rotated at their slot numbers).  src may be the
-// pot rows themselves (rows that a host copy already put in place): the plain copy then rewrites them as they are.
+template <typename T, bool kInterleaved>
+__device__ __forceinline__ void rope_two_vectors(const uint4 &a, const uint4 &b, int g, int half_vecs, int pos,
+                                                 const T *__restrict__ cos_t, const T *__restrict__ sin_t,
+                                                 uint4 &a_out, uint4 &b_out)
+{
+    RopeTab<T, kInterleaved> tab;
+    tab.load(g, half_vecs, pos, cos_t, sin_t);
+    rope_apply<T, kInterleaved>(a, b, g, half_vecs, tab, a_out, b_out);
+}
+
+// grid (pieces, units, 2 or 1).  z = 0: src: key rows of unit y at src + y * src_unit_vecs, n rows of row_vecs vectors;
+// the rows go to pot rows first_row ... of potK (unchanged) and potKrot (rotated at their slot numbers).  src may be
+// the pot rows themselves (rows that a host copy already put in place): the plain copy then rewrites them as they
+// are.  z = 1: the value rows, a plain copy as in append_kernel (srcV is [units][n * row_vecs]).
 template <typename T, bool kInterleaved>
 __global__ void __launch_bounds__(kMoveThreads)
 append_rope_kernel(const uint4 *__restrict__ src, size_t src_unit_vecs, uint4 *potK, uint4 *__restrict__ potKrot,
-                   const T *__restrict__ cos_t, const T *__restrict__ sin_t, int n, int row_vecs, size_t unit_vecs, int first_row)
+                   const T *__restrict__ cos_t, const T *__restrict__ sin_t, int n, int row_vecs, size_t unit_vecs, int first_row,
+                   const uint4 *__restrict__ srcV, uint4 *__restrict__ potV)
 {
+    if (blockIdx.z == 1) {
+        const size_t n_vecs = (size_t)n * row_vecs;
+        append_body(srcV + (size_t)blockIdx.y * n_vecs, potV + (size_t)blockIdx.y * unit_vecs + (size_t)first_row * row_vecs,
+                    n_vecs, blockIdx.x, gridDim.x);
+        return;
+    }
     const int half_vecs = row_vecs / 2;
     const uint4 *s = src + (size_t)blockIdx.y * src_unit_vecs;
     uint4 *dk = potK + (size_t)blockIdx.y * unit_vecs + (size_t)first_row * row_vecs;
     uint4 *dr = potKrot + (size_t)blockIdx.y * unit_vecs + (size_t)first_row * row_vecs;
     const size_t items = (size_t)n * half_vecs, stride = (size_t)gridDim.x * kMoveThreads;
-    for (size_t it = (size_t)blockIdx.x * kMoveThreads + threadIdx.x; it < items; it += stride) {
+    size_t it = (size_t)blockIdx.x * kMoveThreads + threadIdx.x;
+    for (; it + stride < items; it += 2 * stride) {  // two items (four loads) in flight
+        size_t ia[2], ib[2];
+        int g[2], r[2];
+        uint4 a[2], b[2];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const size_t item = it + u * stride;
+            r[u] = (int)(item / half_vecs);
+            g[u] = (int)(item - (size_t)r[u] * half_vecs);
+            ia[u] = (size_t)r[u] * row_vecs + g[u];
+            ib[u] = ia[u] + half_vecs;
+            a[u] = s[ia[u]];
+            b[u] = s[ib[u]];
+        }
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            uint4 ra, rb;
+            rope_two_vectors<T, kInterleaved>(a[u], b[u], g[u], half_vecs, first_row + r[u], cos_t, sin_t, ra, rb);
+            dk[ia[u]] = a[u];
+            dk[ib[u]] = b[u];
+            dr[ia[u]] = ra;
+            dr[ib[u]] = rb;
+        }
+    }
+    for (; it < items; it += stride) {
         const int r = (int)(it / half_vecs), g = (int)(it - (size_t)r * half_vecs);
         const size_t ia = (size_t)r * row_vecs + g, ib = ia + half_vecs;
         const uint4 a = s[ia], b = s[ib];
@@ -128,15 +190,25 @@ append_rope_kernel(const uint4 *__restrict__ src, size_t src_unit_vecs, uint4 *p
     }
 }
 
-// In-place gather of the unrotated keys with the rotated copy written beside it.  grid (slices, units).  A block
+// In-place gather of the unrotated keys with the rotated copy written beside it.
+// grid (max(k_slices, v_slices), units, 2).  For z = 0 a block
 // owns the vector pairs (g, g + row_vecs / 2) with g in [slice * slice_vecs, (slice + 1) * slice_vecs) of every row
 // of one unit; the walk over the rows is compact_kernel's (ascending chunks, read - barrier - write), which is
 // safe in place because idx[r] >= r.  The rotated copy is only written, never read.
+// z = 1 (if launched): the value rows, compact_kernel's walk with its own slicing (v_slices slices of v_slice_vecs).
 template <typename T, bool kInterleaved>
 __global__ void __launch_bounds__(kMoveThreads)
 compact_rope_kernel(uint4 *potK, uint4 *__restrict__ potKrot, const T *__restrict__ cos_t, const T *__restrict__ sin_t,
-                    const int32_t *__restrict__ idx, int keep, int N, int row_vecs, int slice_vecs, size_t unit_vecs, int *status)
+                    const int32_t *__restrict__ idx, int keep, int N, int row_vecs, int k_slices, int slice_vecs, size_t unit_vecs,
+                    int *status, uint4 *potV, int v_slices, int v_slice_vecs)
 {
+    if (blockIdx.z == 1) {
+        if ((int)blockIdx.x < v_slices)
+            compact_body(potV + (size_t)blockIdx.y * unit_vecs + (size_t)blockIdx.x * v_slice_vecs, idx + (size_t)blockIdx.y * keep,
+                         keep, N, row_vecs, v_slice_vecs, status);
+        return;
+    }
+    if ((int)blockIdx.x >= k_slices) return;
     const int half_vecs = row_vecs / 2;
     uint4 *base = potK + (size_t)blockIdx.y * unit_vecs;
     uint4 *rbase = potKrot + (size_t)blockIdx.y * unit_vecs;
@@ -170,6 +242,8 @@ compact_rope_kernel(uint4 *potK, uint4 *__restrict__ potKrot, const T *__restric
             const int r = r0 + i * rows_per_pass + my_row;
             if (src[i] >= 0) {
                 uint4 ra, rb;
+                // the table vectors are fetched here, not with the rows: holding them across the barrier costs a
+                // third of the resident blocks (measured: 164 us against 142 us on the 32-layer workload)
                 rope_two_vectors<T, kInterleaved>(ta[i], tb[i], g, half_vecs, r, cos_t, sin_t, ra, rb);
                 base[(size_t)r * row_vecs + g] = ta[i];
                 base[(size_t)r * row_vecs + g + half_vecs] = tb[i];
