@@ -35,10 +35,11 @@ def _load():
                                       C.c_int, C.c_int, C.c_int, C.c_size_t, dp, ip, bp, bp]
         lib.ora_token_novelty.argtypes = [dp, ip, C.c_long, C.c_int, dp]
         lib.ora_rope_rows.argtypes = [C.c_void_p, C.c_void_p, ip, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_int]
+        lib.ora_decode_attention.argtypes = [dp, dp, dp, C.c_int, C.c_int, C.c_int, dp, dp]
         lib.ora_set_threads.argtypes = [C.c_int]
         lib.ora_max_threads.restype = C.c_int
         for f in (lib.ora_nuc_top, lib.ora_cap_scores, lib.ora_select, lib.ora_gather,
-                  lib.ora_cycle, lib.ora_set_threads, lib.ora_cap_scores_incl, lib.ora_cycle_cap, lib.ora_token_novelty, lib.ora_rope_rows):
+                  lib.ora_cycle, lib.ora_set_threads, lib.ora_cap_scores_incl, lib.ora_cycle_cap, lib.ora_token_novelty, lib.ora_rope_rows, lib.ora_decode_attention):
             f.restype = None
         _lib = lib
     return _lib
@@ -87,6 +88,25 @@ def rope_rows(rows, pos, cos_t, sin_t, interleaved: bool = False) -> np.ndarray:
         _load().ora_rope_rows(flat_in[i].ctypes.data, flat_out[i].ctypes.data, _p(pos, C.c_int), n, d,
                               int(rows.dtype == np.float32), cos_t.ctypes.data, sin_t.ctypes.data, int(interleaved))
     return out
+
+
+def decode_attention(q, K, V, n: int | None = None):
+    """Generation over the pot: q [L][B][Hq][d], K, V [L][B][Hkv][rows][d] in storage dtype (the first ``n`` rows
+    count; K as the queries should see it, i.e. rotated if the pot is in rotary mode).  Query head h reads the
+    rows of KV head h // G.  Returns (out [L][B][Hq][d], lse [L][B][Hq]) in float64."""
+    L, B, Hq, d = q.shape
+    Hkv = K.shape[2]
+    n = K.shape[3] if n is None else n
+    G = Hq // Hkv
+    qd = widen_storage(q).reshape(L * B * Hkv, G, d)
+    Kd = widen_storage(np.ascontiguousarray(K[:, :, :, :n])).reshape(L * B * Hkv, n, d)
+    Vd = widen_storage(np.ascontiguousarray(V[:, :, :, :n])).reshape(L * B * Hkv, n, d)
+    out = np.empty((L * B * Hkv, G, d), dtype=np.float64)
+    lse = np.empty((L * B * Hkv, G), dtype=np.float64)
+    for u in range(L * B * Hkv):
+        _load().ora_decode_attention(_p(np.ascontiguousarray(qd[u]), C.c_double), _p(Kd[u], C.c_double), _p(Vd[u], C.c_double),
+                                     G, n, d, _p(out[u], C.c_double), _p(lse[u], C.c_double))
+    return out.reshape(L, B, Hq, d), lse.reshape(L, B, Hq)
 
 
 def token_novelty(logits, labels) -> np.ndarray:

@@ -23,6 +23,9 @@
  *                    take probability mass from the pot columns
  *   ora_rope_rows    Sec. 3.4 (CR-RoPE): keys are kept without rotary embedding and get it
  *                    at their position inside the pot, 0 .. len-1
+ *   ora_decode_attention  generation over the pot (Sec. 3.3.1 notes that the heads keep different
+ *                    tokens; Sec. 4.5 measures generation at a fixed pot): plain softmax attention
+ *                    of one new query per head over the unit's own rows
  *   ora_cycle        the four steps over every (layer, stream, kv-head) unit
  *   ora_cycle_cap    the same with the CaP-inclusive scores
  *
@@ -58,6 +61,8 @@
  * Rotary rows: position 0 is the identity, exact small cases, complex multiplication in
  * double precision, pair norms, the score of a rotated query and key depends on the
  * position difference only, the two pairings are one channel permutation apart.
+ * Decode attention: one key returns its value, equal keys the mean value, library attention
+ * and log-sum-exp, slot permutation invariance.
  */
 #include <math.h>
 #include <stdint.h>
@@ -225,6 +230,37 @@ void ora_rope_rows(const void *in, void *out, const int *pos, int n, int d, int 
             ora_store(out, ihi, is_f32, fmaf(hi, cs, t2));
         }
     }
+}
+
+/*
+ * Attention of G new queries (the query heads of one KV head, [G][d]) over the N rows of a unit:
+ * out[h] = sum_j softmax_j(q_h . k_j / sqrt(d)) v_j, lse[h] = log sum_j exp(q_h . k_j / sqrt(d))
+ * (lse lets a caller merge this with attention over tokens that are not in the pot).
+ */
+void ora_decode_attention(const double *Q, const double *K, const double *V, int G, int N, int d,
+                          double *out, double *lse)
+{
+    double *s = (double *)malloc(sizeof(double) * (size_t)(N > 0 ? N : 1));
+    const double scale = 1.0 / sqrt((double)d);
+    for (int h = 0; h < G; ++h) {
+        const double *q = Q + (size_t)h * d;
+        double m = -INFINITY;
+        for (int j = 0; j < N; ++j) {
+            double acc = 0.0;
+            for (int c = 0; c < d; ++c) acc += q[c] * K[(size_t)j * d + c];
+            s[j] = acc * scale;
+            if (s[j] > m) m = s[j];
+        }
+        double Z = 0.0;
+        for (int j = 0; j < N; ++j) { s[j] = exp(s[j] - m); Z += s[j]; }
+        for (int c = 0; c < d; ++c) {
+            double o = 0.0;
+            for (int j = 0; j < N; ++j) o += (s[j] / Z) * V[(size_t)j * d + c];
+            out[(size_t)h * d + c] = o;
+        }
+        if (lse) lse[h] = m + log(Z);
+    }
+    free(s);
 }
 
 /*

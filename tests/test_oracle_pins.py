@@ -450,3 +450,38 @@ def test_cycle_with_rope_scores_rotated_keys_and_moves_unrotated_rows():
         assert (out["K"][unit] == src).all()                                           # unrotated rows move
         assert (out["K_rot"][unit] == oracle.rope_rows(src, np.arange(keep), cos_t, sin_t)).all()   # new positions
     assert not np.allclose(out["u"], oracle.cycle(Q, K, V, aux, keep, T)["u"])
+
+
+# ---------------------------------------------------------------- generation over the pot
+def test_decode_attention_closed_forms_and_library():
+    torch = pytest.importorskip("torch")
+    from scipy.special import logsumexp
+    g = rnd(80)
+    L, B, Hq, Hkv, d, N = 2, 2, 6, 2, 16, 37
+    q = g.standard_normal((L, B, Hq, d)).astype(np.float32) * 2
+    K = g.standard_normal((L, B, Hkv, N, d)).astype(np.float32)
+    V = g.standard_normal((L, B, Hkv, N, d)).astype(np.float32)
+    out, lse = oracle.decode_attention(q, K, V)
+    G = Hq // Hkv
+    for l in range(L):
+        for b in range(B):
+            for h in range(Hq):
+                kv = h // G                                       # query head h reads KV head h // G
+                s = K[l, b, kv].astype(np.float64) @ q[l, b, h].astype(np.float64) / np.sqrt(d)
+                np.testing.assert_allclose(lse[l, b, h], logsumexp(s), rtol=1e-12)
+                ref = torch.nn.functional.scaled_dot_product_attention(
+                    torch.from_numpy(q[l, b, h].astype(np.float64))[None, None, :],
+                    torch.from_numpy(K[l, b, kv].astype(np.float64))[None], torch.from_numpy(V[l, b, kv].astype(np.float64))[None])
+                np.testing.assert_allclose(out[l, b, h], ref[0, 0].numpy(), rtol=1e-10, atol=1e-12)
+    # one row: its value comes back; equal keys: the mean value; only the first n rows count
+    o1, l1 = oracle.decode_attention(q, K, V, n=1)
+    for h in range(Hq):
+        np.testing.assert_allclose(o1[0, 0, h], V[0, 0, h // G, 0], rtol=1e-14)
+    Ke = np.broadcast_to(K[:, :, :, :1], K.shape).copy()
+    oe, le = oracle.decode_attention(q, Ke, V)
+    np.testing.assert_allclose(oe[1, 1, 4], V[1, 1, 4 // G].astype(np.float64).mean(axis=0), rtol=1e-12)
+    np.testing.assert_allclose(le - np.log(N), oracle.decode_attention(q, Ke, V, n=1)[1], rtol=1e-12)
+    perm = g.permutation(N)                                       # the order of the slots does not matter
+    op, lp = oracle.decode_attention(q, K[:, :, :, perm], V[:, :, :, perm])
+    np.testing.assert_allclose(op, out, rtol=1e-11, atol=1e-13)
+    np.testing.assert_allclose(lp, lse, rtol=1e-12)
