@@ -199,6 +199,21 @@ int ipot_nuc_scores(ipot_t *pot, const void *logits, int logits_dtype, long long
                     int slot0);
 
 /*
+ * Generation over the pot.  After a cycle the heads of a layer hold different tokens (the CaP score is per
+ * head, Sec. 3.3.1), so each (layer, stream, kv-head) unit is its own cache; Sec. 4.5 measures generation
+ * at a fixed pot.  For one new token: query head h attends to rows [0, len) of the unit of KV head
+ * h / (Hq / Hkv):  out_h = sum_j softmax_j(q_h . k_j / sqrt(d)) v_j.
+ *   q   : device, [layers][batch][Hq][d], pot dtype, 16-byte aligned (in rotary mode: rotated at the new
+ *         token's position by the caller; the keys read are then the rotated copy).  Caller-owned.
+ *   out : device, [layers][batch][Hq][d] fp32, normalised.
+ *   lse : device, [layers][batch][Hq] fp32, or NULL: log sum_j exp(q_h . k_j / sqrt(d)), with which a
+ *         caller merges this result with attention over tokens that are not in the pot.
+ * Supported: Hq / Hkv in {1, 2, 4, 8} and rows of 64, 128, 256 or 512 bytes (else IPOT_E_INVALID).
+ * Requires len >= 1 (IPOT_E_STATE).  Asynchronous on the pot's stream; the pot is not changed.
+ */
+int ipot_decode_attention(ipot_t *pot, const void *q, float *out, float *lse);
+
+/*
  * Context-reset rotary embedding (Sec. 3.4): the pot keeps its keys WITHOUT rotary embedding and every
  * slot j carries position j, so positions run 0 .. len-1 again after each cycle.  With this mode on, the
  * K rows passed to ipot_append_chunk are unrotated keys; the library maintains beside them a copy in

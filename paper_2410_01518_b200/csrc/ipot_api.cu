@@ -11,6 +11,7 @@
 
 #include "common.cuh"
 #include "k_cap_self.cuh"
+#include "k_decode.cuh"
 #include "k_move.cuh"
 #include "k_novelty.cuh"
 #include "k_rope.cuh"
@@ -47,6 +48,9 @@ struct ipot {
     int *status;         // sticky device status word
     void *stage_q;       // device staging for the *_host calls
     void *stage_kc;
+    float *dec_partial;  // [units][dec_splits][G][d + 2]: ipot_decode_attention's split results
+    int *dec_counters;   // [units], zero between calls
+    int dec_splits;
     char *nov_scratch;   // scratch of ipot_nuc_scores, grown on demand: 65536 row counters (always zero between
                          // calls), then [tokens][segments] float2
     size_t nov_capacity;  // float2 entries behind the counters
@@ -100,7 +104,7 @@ void free_all(ipot *p)
     tc_plan_destroy(p->tc);
     cudaFree(p->K); cudaFree(p->V); cudaFree(p->Krot); cudaFree(p->scores); cudaFree(p->summed);
     cudaFree(p->row_stats); cudaFree(p->cap_stats); cudaFree(p->nuc_mask); cudaFree(p->idx); cudaFree(p->status);
-    cudaFree(p->stage_q); cudaFree(p->stage_kc); cudaFree(p->stage_aux); cudaFree(p->nov_scratch);
+    cudaFree(p->stage_q); cudaFree(p->stage_kc); cudaFree(p->stage_aux); cudaFree(p->nov_scratch); cudaFree(p->dec_partial); cudaFree(p->dec_counters);
     if (p->ev) {
         for (int i = 0; i < kProfSlots; ++i)
             for (auto &e : p->ev[i]) if (e) cudaEventDestroy(e);
@@ -314,6 +318,37 @@ int launch_novelty(ipot *p, const void *logits, size_t row_stride, const int32_t
 }
 }  // namespace
 
+template <typename T, int G>
+int launch_decode_g(ipot *p, const void *q, float *out, float *lse)
+{
+    constexpr int KT = G <= 4 ? 8 : 4;
+    const int d = p->cfg.d, N = p->len;
+    int splits = p->dec_splits;
+    if (splits > (N + 63) / 64) splits = (N + 63) / 64;  // at least 64 rows per block
+    const size_t smem = decode_smem_bytes(G, d);
+    auto kern = decode_attn_kernel<T, G, KT>;
+    if (smem > 48 * 1024) IPOT_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    dim3 grid(splits, p->units);
+    kern<<<grid, kDecThreads, smem, p->stream>>>((const T *)score_keys(p), (const T *)p->V, (const T *)q, out, lse, p->dec_partial,
+                                                 p->dec_counters, N, d, p->row_bytes / 16, (size_t)p->cfg.pot_size * d,
+                                                 (float)(1.4426950408889634 / std::sqrt((double)d)));
+    p->launches += 1;
+    IPOT_CUDA(cudaGetLastError());
+    return IPOT_OK;
+}
+
+template <typename T>
+int launch_decode(ipot *p, const void *q, float *out, float *lse)
+{
+    switch (p->G) {
+    case 1: return launch_decode_g<T, 1>(p, q, out, lse);
+    case 2: return launch_decode_g<T, 2>(p, q, out, lse);
+    case 4: return launch_decode_g<T, 4>(p, q, out, lse);
+    case 8: return launch_decode_g<T, 8>(p, q, out, lse);
+    default: return IPOT_E_INVALID;
+    }
+}
+
 extern "C" {
 
 int ipot_create(int pot_size, int keep, int layers, int Hq, int Hkv, int d, ipot_t **out)
@@ -363,10 +398,15 @@ int ipot_create_ex(const ipot_config_t *cfg, ipot_t **out)
     alloc((void **)&p->nuc_mask, (size_t)cfg->batch * cfg->pot_size);
     alloc((void **)&p->idx, (size_t)p->units * cfg->keep * 4);
     alloc((void **)&p->status, 16);
+    p->dec_splits = (8 * p->sm_count + p->units - 1) / p->units;
+    if (p->dec_splits > 64) p->dec_splits = 64;
+    if (p->dec_splits < 1) p->dec_splits = 1;
+    alloc((void **)&p->dec_partial, (size_t)p->units * p->dec_splits * p->G * (cfg->d + 2) * sizeof(float));
+    alloc((void **)&p->dec_counters, (size_t)p->units * sizeof(int));
     alloc(&p->stage_q, (size_t)p->units * maxM * p->row_bytes);
     alloc(&p->stage_kc, (size_t)p->units * cfg->max_cap_rows * p->row_bytes);
     alloc((void **)&p->stage_aux, (size_t)cfg->batch * cfg->pot_size * 4);
-    if (ok) ok = cudaMemset(p->status, 0, 16) == cudaSuccess;
+    if (ok) ok = cudaMemset(p->status, 0, 16) == cudaSuccess && cudaMemset(p->dec_counters, 0, (size_t)p->units * sizeof(int)) == cudaSuccess;
     if (!ok) {
         cudaGetLastError();
         free_all(p);
@@ -564,7 +604,7 @@ int ipot_nuc_scores(ipot_t *p, const void *logits, int logits_dtype, long long r
     const size_t need = rows * ((vocab + kNovSegElems - 1) / kNovSegElems);
     if (!p->nov_scratch || need > p->nov_capacity) {  // first use or a larger shape: the only allocation outside ipot_create
         IPOT_CUDA(cudaStreamSynchronize(p->stream));
-        cudaFree(p->nov_scratch);
+        cudaFree(p->nov_scratch); cudaFree(p->dec_partial); cudaFree(p->dec_counters);
         p->nov_scratch = nullptr;
         p->nov_capacity = 0;
         if (cudaMalloc((void **)&p->nov_scratch, kNovCounterBytes + need * sizeof(float2)) != cudaSuccess) {
@@ -577,6 +617,17 @@ int ipot_nuc_scores(ipot_t *p, const void *logits, int logits_dtype, long long r
     return logits_dtype == IPOT_F32
                ? launch_novelty<float>(p, logits, (size_t)row_stride, labels, n_tokens, vocab, aux_out, (size_t)aux_stride, slot0)
                : launch_novelty<__nv_bfloat16>(p, logits, (size_t)row_stride, labels, n_tokens, vocab, aux_out, (size_t)aux_stride, slot0);
+}
+
+int ipot_decode_attention(ipot_t *p, const void *q, float *out, float *lse)
+{
+    if (!p || !q || !out || !aligned16(q) || (reinterpret_cast<uintptr_t>(out) & 3u) || (reinterpret_cast<uintptr_t>(lse) & 3u))
+        return IPOT_E_INVALID;
+    const int lpk = p->row_bytes / 16;
+    if (p->row_bytes % 16 || (lpk != 4 && lpk != 8 && lpk != 16 && lpk != 32)) return IPOT_E_INVALID;
+    if (p->G != 1 && p->G != 2 && p->G != 4 && p->G != 8) return IPOT_E_INVALID;
+    if (p->len < 1) return IPOT_E_STATE;
+    return p->cfg.dtype == IPOT_F32 ? launch_decode<float>(p, q, out, lse) : launch_decode<__nv_bfloat16>(p, q, out, lse);
 }
 
 int ipot_enable_rope(ipot_t *p, const void *cos_table, const void *sin_table, int pairing)

@@ -31,6 +31,7 @@ SYMBOLS = [
     "ipot_kernel_ms", "ipot_launch_count", "ipot_strerror", "ipot_cap_scores_noalloc",
     "ipot_score_and_compress_cap", "ipot_score_only_cap", "ipot_score_and_compress_cap_host",
     "ipot_nuc_scores", "ipot_enable_rope", "ipot_view_rope",
+    "ipot_decode_attention",
 ]
 
 
@@ -78,6 +79,7 @@ def lib() -> C.CDLL:
         L.ipot_score_only_cap.argtypes = [vp, vp, vp, ip, vp]
         L.ipot_score_and_compress_cap_host.argtypes = [vp, vp, vp, ip, vp, vp]
         L.ipot_nuc_scores.argtypes = [vp, vp, ip, C.c_longlong, vp, ip, ip, vp, C.c_longlong, ip]
+        L.ipot_decode_attention.argtypes = [vp, vp, vp, vp]
         L.ipot_enable_rope.argtypes = [vp, vp, vp, ip]
         L.ipot_view_rope.argtypes = [vp, C.POINTER(vp)]
         L.ipot_view.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(ip)]
@@ -189,6 +191,10 @@ def ipot_score_only_cap(h, Q_cap, K_cap, cap_rows, aux_scores=None) -> None:
 def ipot_nuc_scores(h, logits, logits_dtype, row_stride, labels, n_tokens, vocab, aux_out, aux_stride, slot0) -> None:
     _check(lib().ipot_nuc_scores(h, _ptr(logits), logits_dtype, row_stride, _ptr(labels), n_tokens, vocab,
                                  _ptr(aux_out), aux_stride, slot0), "ipot_nuc_scores")
+
+
+def ipot_decode_attention(h, q, out, lse=None) -> None:
+    _check(lib().ipot_decode_attention(h, _ptr(q), _ptr(out), _ptr(lse)), "ipot_decode_attention")
 
 
 def ipot_enable_rope(h, cos_table, sin_table, pairing) -> None:
