@@ -32,6 +32,8 @@ from paper_2410_01518_b200 import inputs  # noqa: E402
 WORKLOADS = {"cfg2": 2, "cfg3": 3, "cfg4": 4, "cfg5": 5}
 # the token-novelty producer alone (Eq. 3): (vocabulary, new tokens per step), bf16 logits, one stream
 NOVELTY_WORKLOADS = {"nuc32k": (32000, 2048), "nuc128k": (128256, 2048)}
+# generation over a full pot alone: one new token's attention over all layers' units, configs[cfg - 1] shape
+DECODE_WORKLOADS = {"decode3": 3, "decode4": 4, "decode5": 5}
 RING = 4  # distinct chunks / query sets cycled through
 
 
@@ -173,6 +175,135 @@ def run_reference(args, cfg):
     print(json.dumps(line))
 
 
+def run_decode(args):
+    """Generation over the pot alone: a step is one ipot_decode_attention call over every unit of a full pot."""
+    cfg = inputs.CONFIGS[DECODE_WORKLOADS[args.workload]]
+    if args.layers > 0:
+        cfg = cfg.with_layers(args.layers)
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    N = cfg.pot_size
+    workload = (f"configs[{cfg.cfg_id - 1}] {cfg.name}: one new token attends to the full pot "
+                f"({cfg.units} units x {N} rows)")
+    rng = np.random.default_rng(cfg.seed)
+    qs = [inputs.store(rng.standard_normal((cfg.layers, cfg.batch, cfg.Hq, cfg.d), dtype=np.float32), cfg.dtype) for _ in range(RING)]
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        import oracle
+        small = cfg.with_layers(1)
+        K, V = inputs.make_kv(small, N)
+        q1 = qs[0][:1]
+        for _ in range(args.warmup):
+            oracle.decode_attention(q1, K[:, :, :, :64], V[:, :, :, :64])
+        times = []
+        for _ in range(args.steps):
+            t0 = time.perf_counter()
+            oracle.decode_attention(q1, K, V)
+            times.append(time.perf_counter() - t0)
+        ms = float(np.mean(times)) * 1e3 * cfg.layers
+        print(json.dumps({
+            "impl": "reference", "metric": "decode_tokens_per_s", "value": cfg.batch * 1e3 / ms, "unit": "tokens/s", "n_gpus": 1,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": {"workload": workload},
+            "cpu_baseline": {"value": cfg.batch * 1e3 / ms, "unit": "tokens/s", "cores": 1, "kind": "oracle",
+                             "sample": f"1 of {cfg.layers} layers per step, extrapolated"},
+            "e2e": {"value": cfg.batch * 1e3 / ms, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2410_01518_b200 import ipot
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the compression path has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    tdt = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
+
+    def dev(a):
+        t = torch.from_numpy(a.view(np.int16) if a.dtype == np.uint16 else a).cuda()
+        return t.view(tdt) if a.dtype == np.uint16 else t
+
+    h = ipot.ipot_create_ex(cfg.pot_size, cfg.keep, cfg.layers, cfg.Hq, cfg.Hkv, cfg.d, batch=cfg.batch,
+                            dtype=ipot.IPOT_BF16 if cfg.dtype == "bf16" else ipot.IPOT_F32, nuc_slots=cfg.nuc_slots, max_cap_rows=1)
+    stream = torch.cuda.current_stream()
+    ipot.ipot_set_stream(h, stream.cuda_stream)
+    K, V = inputs.make_kv(cfg, N)
+    ipot.ipot_append_chunk(h, dev(K), dev(V), N)
+    dq = [dev(a) for a in qs]
+    hq = [torch.from_numpy(a.view(np.int16) if a.dtype == np.uint16 else a).pin_memory() for a in qs]
+    stage_q = torch.empty_like(dq[0])
+    out = torch.empty((cfg.layers, cfg.batch, cfg.Hq, cfg.d), device="cuda")
+    out_host = torch.empty(out.shape, dtype=torch.float32).pin_memory()
+    pot_bytes = 2 * cfg.units * N * cfg.d * cfg.elem_bytes
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda") if pot_bytes <= 126e6 else None
+
+    def step_dev(i):
+        if flush is not None:
+            flush.add_(1)
+        ipot.ipot_decode_attention(h, dq[i % RING], out)
+
+    def step_host(i):
+        (stage_q.view(torch.int16) if cfg.dtype == "bf16" else stage_q).copy_(hq[i % RING], non_blocking=True)
+        ipot.ipot_decode_attention(h, stage_q, out)
+        out_host.copy_(out, non_blocking=True)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(step, steps, warmup, sampler=None):
+        for i in range(warmup):
+            step(i)
+        barrier()
+        if sampler:
+            sampler.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        l0 = ipot.ipot_launch_count(h)
+        e0.record(stream)
+        for i in range(steps):
+            step(warmup + i)
+        e1.record(stream)
+        barrier()
+        clocks = sampler.stop() if sampler else None
+        rate, ms_step = whole_job_rate(e0.elapsed_time(e1), steps, world, "cuda")
+        return rate * cfg.batch, ms_step, ipot.ipot_launch_count(h) - l0, clocks
+
+    value, ms_step, launches, clocks = timed(step_dev, args.steps, args.warmup, ClockSampler(local))
+    e2e_value, _, _, _ = timed(step_host, max(3, min(args.steps, 200)), 3)
+    assert ipot.ipot_sync_status(h) == 0, "device status is not clean"
+    pk = peaks()
+    algo = pot_bytes + cfg.layers * cfg.batch * cfg.Hq * cfg.d * (cfg.elem_bytes + 4)   # K and V once, q in, out
+    roof = {"kernel": "decode_attn_kernel", "bound": "hbm", "achieved": algo / (ms_step * 1e-3) / 1e9, "peak": pk["hbm_gbs"],
+            "unit": "GB/s", "peak_source": pk["source"], "traffic": None}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    line = {
+        "metric": "decode_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": workload, "l2": "inputs_larger_than_l2" if flush is None else "l2_flushed_between_steps"},
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": qs[0].nbytes, "d2h_bytes_per_step": out_host.numel() * 4},
+        "gpu_launches": launches, "roofline": roof,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        t0 = time.perf_counter()
+        oracle.decode_attention(qs[0][:1], K[:1], V[:1])
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": cfg.batch / (dt * cfg.layers), "unit": "tokens/s", "cores": 1, "kind": "oracle",
+                                "sample": f"1 of {cfg.layers} layers in {dt:.2f} s, extrapolated"}
+    if rank == 0:
+        print(json.dumps(line))
+    ipot.ipot_destroy(h)
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def run_novelty(args):
     """The novelty producer alone: a step turns one chunk's logits into per-token novelty scores."""
     V, n = NOVELTY_WORKLOADS[args.workload]
@@ -307,7 +438,7 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg3", choices=sorted(WORKLOADS) + sorted(NOVELTY_WORKLOADS))
+    ap.add_argument("--workload", default="cfg3", choices=sorted(WORKLOADS) + sorted(NOVELTY_WORKLOADS) + sorted(DECODE_WORKLOADS))
     ap.add_argument("--scorer", default="auto", choices=["auto", "simt", "tensor"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cap-keys", action="store_true",
@@ -319,6 +450,9 @@ def main():
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.workload in NOVELTY_WORKLOADS:
         run_novelty(args)
+        return
+    if args.workload in DECODE_WORKLOADS:
+        run_decode(args)
         return
     cfg = inputs.CONFIGS[WORKLOADS[args.workload]]
     if args.layers > 0:

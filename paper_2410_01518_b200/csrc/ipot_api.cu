@@ -321,12 +321,12 @@ int launch_novelty(ipot *p, const void *logits, size_t row_stride, const int32_t
 template <typename T, int G>
 int launch_decode_g(ipot *p, const void *q, float *out, float *lse)
 {
-    constexpr int KT = G <= 4 ? 8 : 4;
     const int d = p->cfg.d, N = p->len;
     int splits = p->dec_splits;
-    if (splits > (N + 63) / 64) splits = (N + 63) / 64;  // at least 64 rows per block
+    const int tile_keys = kDecStageVecs / (p->row_bytes / 16);
+    if (splits > (N + tile_keys - 1) / tile_keys) splits = (N + tile_keys - 1) / tile_keys;  // at least one stage of rows per block
     const size_t smem = decode_smem_bytes(G, d);
-    auto kern = decode_attn_kernel<T, G, KT>;
+    auto kern = decode_attn_kernel<T, G>;
     if (smem > 48 * 1024) IPOT_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     dim3 grid(splits, p->units);
     kern<<<grid, kDecThreads, smem, p->stream>>>((const T *)score_keys(p), (const T *)p->V, (const T *)q, out, lse, p->dec_partial,
@@ -398,7 +398,7 @@ int ipot_create_ex(const ipot_config_t *cfg, ipot_t **out)
     alloc((void **)&p->nuc_mask, (size_t)cfg->batch * cfg->pot_size);
     alloc((void **)&p->idx, (size_t)p->units * cfg->keep * 4);
     alloc((void **)&p->status, 16);
-    p->dec_splits = (8 * p->sm_count + p->units - 1) / p->units;
+    p->dec_splits = (6 * p->sm_count + p->units - 1) / p->units;
     if (p->dec_splits > 64) p->dec_splits = 64;
     if (p->dec_splits < 1) p->dec_splits = 1;
     alloc((void **)&p->dec_partial, (size_t)p->units * p->dec_splits * p->G * (cfg->d + 2) * sizeof(float));
