@@ -208,7 +208,10 @@ int ipot_nuc_scores(ipot_t *pot, const void *logits, int logits_dtype, long long
  *   out : device, [layers][batch][Hq][d] fp32, normalised.
  *   lse : device, [layers][batch][Hq] fp32, or NULL: log sum_j exp(q_h . k_j / sqrt(d)), with which a
  *         caller merges this result with attention over tokens that are not in the pot.
- * Supported: Hq / Hkv in {1, 2, 4, 8} and rows of 64, 128, 256 or 512 bytes (else IPOT_E_INVALID).
+ * bf16 pots with d = 64 or 128 and Hq / Hkv <= 8 run on warp-level tensor cores (fp32 accumulation, the
+ * softmax weights kept to 16 mantissa bits); every other supported shape, and every shape after
+ * ipot_set_scorer(IPOT_SCORER_SIMT), uses fp32 FMAs, which needs Hq / Hkv in {1, 2, 4, 8} and rows of 64,
+ * 128, 256 or 512 bytes.  Unsupported shapes: IPOT_E_INVALID.
  * Requires len >= 1 (IPOT_E_STATE).  Asynchronous on the pot's stream; the pot is not changed.
  */
 int ipot_decode_attention(ipot_t *pot, const void *q, float *out, float *lse);

@@ -337,6 +337,25 @@ int launch_decode_g(ipot *p, const void *q, float *out, float *lse)
     return IPOT_OK;
 }
 
+// bf16 rows of 64 or 128 channels: the tensor-core stream
+template <int D>
+int launch_decode_mma(ipot *p, const void *q, float *out, float *lse)
+{
+    const int N = p->len;
+    int splits = p->dec_splits;
+    if (splits > (N + 63) / 64) splits = (N + 63) / 64;  // at least one 16-key tile per warp
+    const size_t smem = decode_mma_smem_bytes(p->G, D);
+    auto kern = decode_attn_mma_kernel<D>;
+    IPOT_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    dim3 grid(splits, p->units);
+    kern<<<grid, kMmaWarps * 32, smem, p->stream>>>((const __nv_bfloat16 *)score_keys(p), (const __nv_bfloat16 *)p->V,
+                                                    (const __nv_bfloat16 *)q, out, lse, p->dec_partial, p->dec_counters, N, p->G,
+                                                    (size_t)p->cfg.pot_size * D, (float)(1.4426950408889634 / std::sqrt((double)D)));
+    p->launches += 1;
+    IPOT_CUDA(cudaGetLastError());
+    return IPOT_OK;
+}
+
 template <typename T>
 int launch_decode(ipot *p, const void *q, float *out, float *lse)
 {
@@ -625,8 +644,11 @@ int ipot_decode_attention(ipot_t *p, const void *q, float *out, float *lse)
         return IPOT_E_INVALID;
     const int lpk = p->row_bytes / 16;
     if (p->row_bytes % 16 || (lpk != 4 && lpk != 8 && lpk != 16 && lpk != 32)) return IPOT_E_INVALID;
-    if (p->G != 1 && p->G != 2 && p->G != 4 && p->G != 8) return IPOT_E_INVALID;
+    if (p->G > 8) return IPOT_E_INVALID;
     if (p->len < 1) return IPOT_E_STATE;
+    if (p->cfg.dtype == IPOT_BF16 && p->scorer != IPOT_SCORER_SIMT && (p->cfg.d == 64 || p->cfg.d == 128))
+        return p->cfg.d == 64 ? launch_decode_mma<64>(p, q, out, lse) : launch_decode_mma<128>(p, q, out, lse);
+    if (p->G != 1 && p->G != 2 && p->G != 4 && p->G != 8) return IPOT_E_INVALID;
     return p->cfg.dtype == IPOT_F32 ? launch_decode<float>(p, q, out, lse) : launch_decode<__nv_bfloat16>(p, q, out, lse);
 }
 

@@ -19,10 +19,11 @@ def make_query(cfg, seed=0):
     return inputs.store(g.standard_normal((cfg.layers, cfg.batch, cfg.Hq, cfg.d), dtype=np.float32) * np.float32(1.5), cfg.dtype)
 
 
-def run_decode(cfg, K, V, q, n, rope=None, with_lse=True):
+def run_decode(cfg, K, V, q, n, rope=None, with_lse=True, scorer=ipot.IPOT_SCORER_AUTO):
     h = make_pot(cfg)
     keep = []
     try:
+        ipot.ipot_set_scorer(h, scorer)   # SIMT: the fp32-FMA stream; otherwise tensor cores where they apply
         if rope is not None:
             keep = [to_dev(rope[0], cfg.dtype), to_dev(rope[1], cfg.dtype)]
             ipot.ipot_enable_rope(h, keep[0], keep[1], ipot.IPOT_ROPE_INTERLEAVED if rope[2] else ipot.IPOT_ROPE_HALF)
@@ -55,17 +56,28 @@ SHAPES = [
     dict(pot_size=512, keep=256, Hq=8, Hkv=1, d=128, dtype="f32", n=1),
     dict(pot_size=5000, keep=2500, Hq=4, Hkv=2, d=32, dtype="f32", n=4999, layers=3),
     dict(pot_size=300, keep=150, Hq=2, Hkv=1, d=128, dtype="bf16", n=65),
+    dict(pot_size=3000, keep=1500, Hq=8, Hkv=1, d=64, dtype="bf16", n=2999, batch=2),      # 8 heads per KV head, 64 channels
+    dict(pot_size=100, keep=50, Hq=1, Hkv=1, d=128, dtype="bf16", n=17),
 ]
 
 
+def test_decode_three_heads_per_kv_head_needs_the_tensor_path():
+    cfg = inputs.small_config(cfg_id=830, pot_size=500, keep=100, nuc_slots=0, cap_rows=1, Hq=6, Hkv=2, d=128, dtype="bf16")
+    K, V = inputs.make_kv(cfg, 500)
+    q = make_query(cfg)
+    out, lse = run_decode(cfg, K, V, q, 500)
+    check(out, lse, *oracle.decode_attention(q, K, V))
+
+
+@pytest.mark.parametrize("scorer", [ipot.IPOT_SCORER_SIMT, ipot.IPOT_SCORER_AUTO])
 @pytest.mark.parametrize("case", range(len(SHAPES)))
-def test_decode_shapes(case):
+def test_decode_shapes(case, scorer):
     kw = dict(SHAPES[case])
     n = kw.pop("n")
     cfg = inputs.small_config(cfg_id=800 + case, nuc_slots=0, cap_rows=1, **kw)
     K, V = inputs.make_kv(cfg, cfg.pot_size)
     q = make_query(cfg)
-    out, lse = run_decode(cfg, K, V, q, n)
+    out, lse = run_decode(cfg, K, V, q, n, scorer=scorer)
     ref_out, ref_lse = oracle.decode_attention(q, K, V, n)
     check(out, lse, ref_out, ref_lse)
 
@@ -123,6 +135,7 @@ def test_decode_after_a_cycle_and_argument_errors():
     odd = inputs.small_config(cfg_id=822, pot_size=64, keep=16, nuc_slots=0, Hq=6, Hkv=2, d=64, dtype="bf16")   # G = 3
     h = make_pot(odd)
     try:
+        ipot.ipot_set_scorer(h, ipot.IPOT_SCORER_SIMT)      # the fp32-FMA stream takes 1, 2, 4 or 8 heads per KV head
         K, V = inputs.make_kv(odd, 64)
         ipot.ipot_append_chunk(h, to_dev(K, "bf16"), to_dev(V, "bf16"), 64)
         o = torch.zeros((1, 1, 6, 64), device="cuda")
