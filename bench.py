@@ -231,6 +231,8 @@ def run_decode(args):
                             dtype=ipot.IPOT_BF16 if cfg.dtype == "bf16" else ipot.IPOT_F32, nuc_slots=cfg.nuc_slots, max_cap_rows=1)
     stream = torch.cuda.current_stream()
     ipot.ipot_set_stream(h, stream.cuda_stream)
+    ipot.ipot_set_scorer(h, {"auto": 0, "simt": 1, "tensor": 2}[args.scorer])
+    tensor_path = args.scorer != "simt" and cfg.dtype == "bf16" and cfg.d in (64, 128)
     K, V = inputs.make_kv(cfg, N)
     ipot.ipot_append_chunk(h, dev(K), dev(V), N)
     dq = [dev(a) for a in qs]
@@ -278,7 +280,7 @@ def run_decode(args):
     assert ipot.ipot_sync_status(h) == 0, "device status is not clean"
     pk = peaks()
     algo = pot_bytes + cfg.layers * cfg.batch * cfg.Hq * cfg.d * (cfg.elem_bytes + 4)   # K and V once, q in, out
-    roof = {"kernel": "decode_attn_kernel", "bound": "hbm", "achieved": algo / (ms_step * 1e-3) / 1e9, "peak": pk["hbm_gbs"],
+    roof = {"kernel": "decode_attn_mma_kernel" if tensor_path else "decode_attn_kernel", "bound": "hbm", "achieved": algo / (ms_step * 1e-3) / 1e9, "peak": pk["hbm_gbs"],
             "unit": "GB/s", "peak_source": pk["source"], "traffic": None}
     roof["frac"] = roof["achieved"] / roof["peak"]
     line = {
