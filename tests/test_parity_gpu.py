@@ -303,3 +303,17 @@ def test_score_only_leaves_the_pot_alone():
         assert abs(u.sum(axis=1) - cfg.G * cfg.cap_rows).max() < 1e-2
     finally:
         ipot.ipot_destroy(h)
+
+
+@pytest.mark.parametrize("scorer", SCORERS)
+def test_largest_pot_the_library_accepts(scorer):
+    """pot_size = 32768 (the create-time limit): 128 slabs per item on the tensor scorer, 512 key tiles on the
+    fp32 scorer; one more slot is refused at create."""
+    cfg = inputs.small_config(cfg_id=290, pot_size=32768, keep=8192, nuc_slots=4096, cap_rows=16, Hq=4, Hkv=1, d=128,
+                              dtype="bf16")
+    t = inputs.make_cycle(cfg)
+    gpu = gpu_cycle(cfg, t, scorer)
+    same, n = compare_cycle(cfg, t, gpu)
+    assert n == cfg.units and same == n
+    rc = ipot.lib().ipot_create(32769, 8192, 1, 4, 1, 128, __import__("ctypes").byref(__import__("ctypes").c_void_p()))
+    assert rc == ipot.IPOT_E_INVALID
