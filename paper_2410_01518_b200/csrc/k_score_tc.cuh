@@ -1,4 +1,4 @@
-// CaP scoring on the 5th-generation tensor cores (Sec. 3.3.1, Eq. 2), bf16, d = 128.
+// CaP scoring on the 5th-generation tensor cores (Sec. 3.3.1, Eq. 2), bf16, d = 128 or 64.
 //
 // Item  = (unit, block of 128 folded query rows): one row-softmax problem over the
 //         unit's N pot keys.
@@ -53,9 +53,9 @@ namespace ipotk {
 constexpr int kTcThreads = 704;      // warp 0: TMA, 1: MMA + TMEM owner, 2-17: pass 1 / pass 2, 18-21: combine
 constexpr int kTcRows = 128;         // query rows per item (TMEM lanes)
 constexpr int kTcSlab = 256;         // keys per task (TMEM columns per buffer)
-constexpr int kTcD = 128;
-constexpr uint32_t kTcQBytes = kTcRows * kTcD * 2;           // 32 KiB
-constexpr uint32_t kTcKBytes = kTcSlab * kTcD * 2;           // 64 KiB
+constexpr int kTcD = 128;            // largest head dimension; 64 uses the first 64-channel half of every tile
+constexpr uint32_t kTcQBytes = kTcRows * kTcD * 2;           // 32 KiB: two halves of 128 rows x 64 channels
+constexpr uint32_t kTcKBytes = kTcSlab * kTcD * 2;           // 64 KiB: two halves of 256 rows x 64 channels
 constexpr uint32_t kTcStageBytes = kTcQBytes + kTcKBytes;    // 96 KiB
 constexpr uint32_t kTcSpinLimit = 1u << 22;                  // try_wait / poll rounds before giving up
 
@@ -78,6 +78,7 @@ struct TcParams {
     float sign;           // +1 or -1: this launch's "fresh" mark
     int *status;
     int N, M, mtiles, slabs, tasks;
+    int dhalves;          // d / 64: 64-channel halves of a tile (1 or 2)
     float scale_log2e;
 };
 
@@ -378,12 +379,14 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                 const int unit = item / prm.mtiles, mt = item - unit * prm.mtiles;
                 const uint32_t b = k & 1, ph = (k >> 1) & 1;
                 mbar_wait(bar(kBarEmpty + b), ph ^ 1, ab, prm.status);
-                mbar_expect_tx(bar(kBarFull + b), kTcStageBytes);
+                mbar_expect_tx(bar(kBarFull + b), (uint32_t)prm.dhalves * (kTcStageBytes / 2));
                 const uint32_t q = base + kTcOffStage + b * kTcStageBytes, kk = q + kTcQBytes;
                 tma_load_3d(q, &mapQ, 0, mt * kTcRows, unit, bar(kBarFull + b));
-                tma_load_3d(q + kTcQBytes / 2, &mapQ, 64, mt * kTcRows, unit, bar(kBarFull + b));
                 tma_load_3d(kk, &mapK, 0, slab * kTcSlab, unit, bar(kBarFull + b));
-                tma_load_3d(kk + kTcKBytes / 2, &mapK, 64, slab * kTcSlab, unit, bar(kBarFull + b));
+                if (prm.dhalves == 2) {
+                    tma_load_3d(q + kTcQBytes / 2, &mapQ, 64, mt * kTcRows, unit, bar(kBarFull + b));
+                    tma_load_3d(kk + kTcKBytes / 2, &mapK, 64, slab * kTcSlab, unit, bar(kBarFull + b));
+                }
             }
         }
         __syncwarp();
@@ -398,11 +401,14 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                 for (uint32_t h = 0; h < 2; ++h) {
                     mbar_wait(bar(kBarTEmpty + 2 * b + h), ph ^ 1, ab, prm.status);
                     tc_fence_after();
+                    for (uint32_t blk = 0; blk < (uint32_t)prm.dhalves; ++blk) {
 #pragma unroll
-                    for (int ks = 0; ks < kTcD / 16; ++ks) {
-                        const uint32_t blk = ks >> 2, off = (ks & 3) * 32;
-                        tc_mma_bf16(tmem + b * kTcSlab + h * 128, smem_desc_sw128(qa + blk * (kTcQBytes / 2) + off),
-                                    smem_desc_sw128(kb + blk * (kTcKBytes / 2) + h * (128 * 128) + off), kTcIdesc, ks > 0 ? 1u : 0u);
+                        for (uint32_t k4 = 0; k4 < 4; ++k4) {
+                            const uint32_t off = k4 * 32;
+                            tc_mma_bf16(tmem + b * kTcSlab + h * 128, smem_desc_sw128(qa + blk * (kTcQBytes / 2) + off),
+                                        smem_desc_sw128(kb + blk * (kTcKBytes / 2) + h * (128 * 128) + off), kTcIdesc,
+                                        (blk | k4) ? 1u : 0u);
+                        }
                     }
                     tc_commit(bar(kBarSFull + 2 * b + h));   // this half's logits are complete
                 }
@@ -595,7 +601,7 @@ inline void tc_plan_init(TcPlan &plan, const ipot_config_t &cfg, const void *, i
 {
     plan.usable = false;
     plan.sm_count = sm_count;
-    if (cfg.dtype != IPOT_BF16 || cfg.d != kTcD) return;
+    if (cfg.dtype != IPOT_BF16 || (cfg.d != 128 && cfg.d != 64)) return;
     int coop = 0, dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop) {
         cudaGetLastError();
@@ -627,16 +633,16 @@ inline void tc_plan_init(TcPlan &plan, const ipot_config_t &cfg, const void *, i
 
 inline bool tc_applicable(TcPlan &plan, const ipot_config_t &cfg, int N, int M)
 {
-    if (!plan.usable || cfg.dtype != IPOT_BF16 || cfg.d != kTcD || N < 1 || M < 1) return false;
+    if (!plan.usable || cfg.dtype != IPOT_BF16 || (cfg.d != 128 && cfg.d != 64) || N < 1 || M < 1) return false;
     const int units = cfg.layers * cfg.batch * cfg.Hkv;
     return units * ((M + kTcRows - 1) / kTcRows) <= plan.max_items && (N + kTcSlab - 1) / kTcSlab <= plan.max_slabs;
 }
 
-// [units][unit_rows][128] bf16, of which `rows` per unit are addressable; box = 64 x box_rows x 1, 128-byte swizzle.
-inline int tc_encode_rows(TcPlan &plan, CUtensorMap *map, const void *ptr, int rows, int units, size_t unit_rows, int box_rows)
+// [units][unit_rows][d] bf16, of which `rows` per unit are addressable; box = 64 x box_rows x 1, 128-byte swizzle.
+inline int tc_encode_rows(TcPlan &plan, CUtensorMap *map, const void *ptr, int d, int rows, int units, size_t unit_rows, int box_rows)
 {
-    cuuint64_t dims[3] = {(cuuint64_t)kTcD, (cuuint64_t)rows, (cuuint64_t)units};
-    cuuint64_t strides[2] = {(cuuint64_t)kTcD * 2, (cuuint64_t)unit_rows * kTcD * 2};
+    cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)rows, (cuuint64_t)units};
+    cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)unit_rows * d * 2};
     cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
     cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = plan.encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(ptr), dims, strides, box, estr,
@@ -652,13 +658,14 @@ inline int tc_launch(TcPlan &plan, const ipot_config_t &cfg, const void *Q, cons
     if (!tc_applicable(plan, cfg, N, M)) return IPOT_E_INVALID;
     const int mtiles = (M + kTcRows - 1) / kTcRows;
     CUtensorMap mapQ, mapK;
-    if (tc_encode_rows(plan, &mapQ, Q, M, units, (size_t)M, kTcRows) != IPOT_OK) return IPOT_E_CUDA;
-    if (tc_encode_rows(plan, &mapK, K, N, units, (size_t)cfg.pot_size, kTcSlab) != IPOT_OK) return IPOT_E_CUDA;
+    if (tc_encode_rows(plan, &mapQ, Q, cfg.d, M, units, (size_t)M, kTcRows) != IPOT_OK) return IPOT_E_CUDA;
+    if (tc_encode_rows(plan, &mapK, K, cfg.d, N, units, (size_t)cfg.pot_size, kTcSlab) != IPOT_OK) return IPOT_E_CUDA;
     TcParams prm;
     prm.scores = scores; prm.part_stride = part_stride; prm.stats = plan.stats; prm.cap_stats = cap_stats; prm.status = status;
     prm.N = N; prm.M = M; prm.mtiles = mtiles; prm.slabs = (N + kTcSlab - 1) / kTcSlab;
     const int items = units * mtiles;
     prm.tasks = items * prm.slabs;
+    prm.dhalves = cfg.d / 64;
     prm.scale_log2e = (float)(1.4426950408889634 / sqrt((double)cfg.d));
     if (items != plan.last_items || prm.slabs != plan.last_slabs) {
         if (cudaMemsetAsync(plan.stats, 0, (size_t)items * prm.slabs * kTcRows * sizeof(float2), stream) != cudaSuccess) {

@@ -58,8 +58,8 @@ SHAPES = [
 @pytest.mark.parametrize("scorer", SCORERS)
 def test_shapes_with_cap_keys(case, scorer):
     cfg = inputs.small_config(cfg_id=500 + case, **SHAPES[case])
-    if scorer == ipot.IPOT_SCORER_TENSOR and not (cfg.dtype == "bf16" and cfg.d == 128):
-        pytest.skip("the tensor scorer takes bf16 with d = 128")
+    if scorer == ipot.IPOT_SCORER_TENSOR and not (cfg.dtype == "bf16" and cfg.d in (64, 128)):
+        pytest.skip("the tensor scorer takes bf16 with d = 128 or 64")
     t = with_cap_keys(cfg)
     gpu = gpu_cycle(cfg, t, scorer)
     same, n = compare_cycle(cfg, t, gpu)

@@ -14,8 +14,8 @@ SCORERS = [ipot.IPOT_SCORER_SIMT, ipot.IPOT_SCORER_TENSOR]
 
 
 def tensor_scorer_applies(cfg, n=None):
-    """The tcgen05 scorer takes bf16 with d = 128 (any pot size the library accepts)."""
-    return cfg.dtype == "bf16" and cfg.d == 128
+    """The tcgen05 scorer takes bf16 with d = 128 or 64 (any pot size the library accepts)."""
+    return cfg.dtype == "bf16" and cfg.d in (64, 128)
 
 
 def test_config1_tiny_f32_all_units():
@@ -68,6 +68,19 @@ def test_small_random_shapes(case, scorer):
     gpu = gpu_cycle(cfg, t, scorer)
     same, n = compare_cycle(cfg, t, gpu)
     assert n == cfg.units and same >= n - 1
+
+
+def test_tensor_scorer_with_64_channel_heads():
+    """d = 64 (one 64-channel half per tile): several slabs and row blocks, ragged tail, against the checker and
+    against the fp32 scorer."""
+    cfg = inputs.small_config(cfg_id=420, pot_size=3000, keep=1400, nuc_slots=700, cap_rows=40, Hq=8, Hkv=2, d=64,
+                              dtype="bf16", layers=3, batch=2)
+    t = inputs.make_cycle(cfg)
+    gpu = gpu_cycle(cfg, t, ipot.IPOT_SCORER_TENSOR, n=2999)
+    same, cnt = compare_cycle(cfg, t, gpu, n=2999)
+    assert cnt == cfg.units and same >= cnt - 1
+    simt = gpu_cycle(cfg, t, ipot.IPOT_SCORER_SIMT, n=2999)
+    np.testing.assert_allclose(gpu[0], simt[0], rtol=2e-5, atol=1e-30)
 
 
 TENSOR_SHAPES = [
