@@ -67,7 +67,7 @@ enum {
 enum {
     IPOT_SCORER_AUTO = 0,   /* tensor-core kernel when the shape allows it, else the SIMT kernel */
     IPOT_SCORER_SIMT = 1,   /* fp32 FMA kernel: any supported shape, f32 or bf16 */
-    IPOT_SCORER_TENSOR = 2  /* tcgen05 kernel: IPOT_E_INVALID if the shape does not allow it */
+    IPOT_SCORER_TENSOR = 2  /* tcgen05 kernel (bf16, d = 64 or 128): IPOT_E_INVALID if the shape does not allow it */
 };
 
 typedef struct {
