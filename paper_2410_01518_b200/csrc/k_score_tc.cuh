@@ -519,12 +519,16 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
             float ls = 0.f;
 #pragma unroll
             for (int i = 0; i < 8; ++i) ls += (cm[i] == -INFINITY) ? 0.f : tstat[(b * 8 + i) * kTcRows + row].y * ex2(cm[i] - ms);
-            st_gpu_f32x2(&prm.stats[((size_t)item * tasks_per_item + slab) * kTcRows + row], ms, ls * sgn);
+            if (tasks_per_item > 1) st_gpu_f32x2(&prm.stats[((size_t)item * tasks_per_item + slab) * kTcRows + row], ms, ls * sgn);
 
             // ---- this row's statistics of every slab of the item; re-read until all carry this launch's mark
             const float2 *st = prm.stats + (size_t)item * tasks_per_item * kTcRows + row;
             float m = -INFINITY, l = 0.f;
-            for (int s0 = 0; s0 < tasks_per_item; s0 += 16) {
+            if (tasks_per_item == 1) {  // the item is this slab: nothing to exchange
+                m = ms;
+                l = ls;
+            }
+            for (int s0 = 0; s0 < (tasks_per_item > 1 ? tasks_per_item : 0); s0 += 16) {
                 float2 sv[16];
                 uint32_t tries = 0;
                 bool fresh;
