@@ -65,9 +65,11 @@ enum {
 
 /* Which scoring kernel ipot_score_and_compress() uses. */
 enum {
-    IPOT_SCORER_AUTO = 0,   /* tensor-core kernel when the shape allows it, else the SIMT kernel */
+    IPOT_SCORER_AUTO = 0,   /* the fastest kernel the shape allows: tcgen05, else warp-level tensor cores, else fp32 FMAs */
     IPOT_SCORER_SIMT = 1,   /* fp32 FMA kernel: any supported shape, f32 or bf16 */
-    IPOT_SCORER_TENSOR = 2  /* tcgen05 kernel (bf16, d = 64 or 128): IPOT_E_INVALID if the shape does not allow it */
+    IPOT_SCORER_TENSOR = 2, /* tcgen05 kernel (bf16, d = 64 or 128): IPOT_E_INVALID if the shape does not allow it */
+    IPOT_SCORER_WARP_MMA = 3 /* warp-level tensor-core kernels (bf16, d a multiple of 16): what AUTO takes for bf16
+                                pots the tcgen05 kernel does not; IPOT_E_INVALID if the shape does not allow it */
 };
 
 typedef struct {
@@ -265,7 +267,7 @@ int ipot_sync_status(ipot_t *pot);
  * over the recorded cycles in milliseconds - ms[0] NuC ranking, ms[1] CaP
  * scoring, ms[2] per-head selection, ms[3] K/V compaction - and starts a new
  * series.  *cycles (may be NULL) = cycles averaged; *scorer_used (may be NULL)
- * = IPOT_SCORER_SIMT or IPOT_SCORER_TENSOR.  STATE if nothing was recorded.
+ * = IPOT_SCORER_SIMT, IPOT_SCORER_TENSOR or IPOT_SCORER_WARP_MMA.  STATE if nothing was recorded.
  */
 int ipot_set_profiling(ipot_t *pot, int on);
 int ipot_kernel_ms(ipot_t *pot, float ms[4], int *cycles, int *scorer_used);

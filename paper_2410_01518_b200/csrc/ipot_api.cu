@@ -15,6 +15,7 @@
 #include "k_move.cuh"
 #include "k_novelty.cuh"
 #include "k_rope.cuh"
+#include "k_score_mma.cuh"
 #include "k_score_simt.cuh"
 #include "k_score_tc.cuh"
 #include "k_select.cuh"
@@ -42,6 +43,7 @@ struct ipot {
     float *summed;       // [units][N]: sum of the partial arrays when there are several
     int max_parts;
     float2 *row_stats;   // [units][max M]
+    float2 *mma_part;    // [kMmaSplits][units][max M]: partial row statistics of the warp-level tensor-core scorer
     float2 *cap_stats;   // [units][max M]: (max, sum) over the CaP's own keys, CaP-inclusive scoring only
     uint8_t *nuc_mask;   // [batch][pot_size]
     int32_t *idx;        // [units][keep]
@@ -70,6 +72,7 @@ struct ipot {
 namespace {
 
 constexpr int kProfSlots = 2048;
+constexpr int kMmaSplits = 8;
 constexpr size_t kNovCounterBytes = (size_t)(kNovMaxRows + 1) * sizeof(int);
 
 #define IPOT_CUDA(call)                                                             \
@@ -103,7 +106,7 @@ void free_all(ipot *p)
 {
     tc_plan_destroy(p->tc);
     cudaFree(p->K); cudaFree(p->V); cudaFree(p->Krot); cudaFree(p->scores); cudaFree(p->summed);
-    cudaFree(p->row_stats); cudaFree(p->cap_stats); cudaFree(p->nuc_mask); cudaFree(p->idx); cudaFree(p->status);
+    cudaFree(p->row_stats); cudaFree(p->mma_part); cudaFree(p->cap_stats); cudaFree(p->nuc_mask); cudaFree(p->idx); cudaFree(p->status);
     cudaFree(p->stage_q); cudaFree(p->stage_kc); cudaFree(p->stage_aux); cudaFree(p->nov_scratch); cudaFree(p->dec_partial); cudaFree(p->dec_counters);
     if (p->ev) {
         for (int i = 0; i < kProfSlots; ++i)
@@ -151,6 +154,31 @@ int launch_simt(ipot *p, const void *Q, const float2 *cap_stats, int M, int N)
     return IPOT_OK;
 }
 
+// bf16 pots with d a multiple of 16 that the tcgen05 kernel does not take: the same two launches on warp-level tensor cores
+int launch_warp_mma(ipot *p, const void *Q, const float2 *cap_stats, int M, int N)
+{
+    const int d = p->cfg.d;
+    const size_t smem = mma_scorer_smem_bytes(d);
+    const float scale_log2e = (float)(1.4426950408889634 / std::sqrt((double)d));
+    const size_t kstride = (size_t)p->cfg.pot_size * d;
+    const int row_tiles = (M + kMsRows - 1) / kMsRows;
+    // the row pass splits the keys so that it launches about four blocks per SM (at most kMmaSplits splits of whole tiles)
+    int nsplit = (4 * p->sm_count + row_tiles * p->units - 1) / (row_tiles * p->units);
+    const int key_tiles = (N + kMsKeys - 1) / kMsKeys;
+    if (nsplit > kMmaSplits) nsplit = kMmaSplits;
+    if (nsplit > key_tiles) nsplit = key_tiles;
+    if (nsplit < 1) nsplit = 1;
+    const int per = ((key_tiles + nsplit - 1) / nsplit) * kMsKeys;
+    dim3 g1(row_tiles, p->units, nsplit), g2(key_tiles, p->units);
+    const __nv_bfloat16 *Qb = (const __nv_bfloat16 *)Q, *Kb = (const __nv_bfloat16 *)score_keys(p);
+    cap_row_stats_mma<<<g1, kMsWarps * 32, smem, p->stream>>>(Qb, Kb, p->mma_part, M, N, d, kstride, scale_log2e, per);
+    cap_column_sums_mma<<<g2, kMsWarps * 32, smem, p->stream>>>(Qb, Kb, p->mma_part, cap_stats, nsplit, p->scores, M, N, d, kstride,
+                                                               scale_log2e);
+    p->launches += 2;
+    IPOT_CUDA(cudaGetLastError());
+    return IPOT_OK;
+}
+
 // Steps 1-2 (and the timing events around them).  On success *parts tells how many
 // partial score arrays the scorer wrote.
 int run_scoring(ipot *p, const void *Q, const void *Kc, int cap_rows, const float *aux, int *parts)
@@ -158,8 +186,10 @@ int run_scoring(ipot *p, const void *Q, const void *Kc, int cap_rows, const floa
     const int N = p->len, T = p->cfg.nuc_slots, M = p->G * cap_rows;
     int scorer = p->scorer;
     const bool tc_ok = tc_applicable(p->tc, p->cfg, N, M);
+    const bool mma_ok = p->cfg.dtype == IPOT_BF16 && p->cfg.d % 16 == 0;
     if (scorer == IPOT_SCORER_TENSOR && !tc_ok) return IPOT_E_INVALID;
-    if (scorer == IPOT_SCORER_AUTO) scorer = tc_ok ? IPOT_SCORER_TENSOR : IPOT_SCORER_SIMT;
+    if (scorer == IPOT_SCORER_WARP_MMA && !mma_ok) return IPOT_E_INVALID;
+    if (scorer == IPOT_SCORER_AUTO) scorer = tc_ok ? IPOT_SCORER_TENSOR : mma_ok ? IPOT_SCORER_WARP_MMA : IPOT_SCORER_SIMT;
 
     cudaEvent_t *ev = (p->profiling && p->ev_used < kProfSlots) ? p->ev[p->ev_used] : nullptr;
     if (ev) IPOT_CUDA(cudaEventRecord(ev[0], p->stream));
@@ -181,6 +211,8 @@ int run_scoring(ipot *p, const void *Q, const void *Kc, int cap_rows, const floa
         rc = tc_launch(p->tc, p->cfg, Q, score_keys(p), cap_stats, p->scores, (size_t)p->units * p->cfg.pot_size, N, M, p->units, p->status,
                        p->stream, parts, &n_launch);
         p->launches += n_launch;
+    } else if (scorer == IPOT_SCORER_WARP_MMA) {
+        rc = launch_warp_mma(p, Q, cap_stats, M, N);
     } else {
         rc = p->cfg.dtype == IPOT_F32 ? launch_simt<float>(p, Q, cap_stats, M, N) : launch_simt<__nv_bfloat16>(p, Q, cap_stats, M, N);
     }
@@ -433,6 +465,7 @@ int ipot_create_ex(const ipot_config_t *cfg, ipot_t **out)
     alloc((void **)&p->summed, score_elems * 4);
     alloc((void **)&p->row_stats, (size_t)p->units * maxM * sizeof(float2));
     alloc((void **)&p->cap_stats, (size_t)p->units * maxM * sizeof(float2));
+    alloc((void **)&p->mma_part, (size_t)kMmaSplits * p->units * maxM * sizeof(float2));
     alloc((void **)&p->nuc_mask, (size_t)cfg->batch * cfg->pot_size);
     alloc((void **)&p->idx, (size_t)p->units * cfg->keep * 4);
     alloc((void **)&p->status, 16);
@@ -455,6 +488,8 @@ int ipot_create_ex(const ipot_config_t *cfg, ipot_t **out)
          cudaFuncSetAttribute(cap_row_stats<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)simt_smem_bytes(256)) == cudaSuccess &&
          cudaFuncSetAttribute(cap_column_sums<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)simt_smem_bytes(256)) == cudaSuccess &&
          cudaFuncSetAttribute(cap_self_stats_bf16, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)self_smem_bytes(256)) == cudaSuccess &&
+         cudaFuncSetAttribute(cap_row_stats_mma, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mma_scorer_smem_bytes(256)) == cudaSuccess &&
+         cudaFuncSetAttribute(cap_column_sums_mma, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mma_scorer_smem_bytes(256)) == cudaSuccess &&
          cudaFuncSetAttribute(nuc_mask_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 32768 * 4) == cudaSuccess &&
          cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 32768 * 4) == cudaSuccess;
     if (!ok) {
@@ -495,7 +530,7 @@ int ipot_set_nuc_slots(ipot_t *p, int T)
 
 int ipot_set_scorer(ipot_t *p, int scorer)
 {
-    if (!p || scorer < IPOT_SCORER_AUTO || scorer > IPOT_SCORER_TENSOR) return IPOT_E_INVALID;
+    if (!p || scorer < IPOT_SCORER_AUTO || scorer > IPOT_SCORER_WARP_MMA) return IPOT_E_INVALID;
     p->scorer = scorer;
     return IPOT_OK;
 }

@@ -19,7 +19,7 @@ from . import build as _build
 IPOT_OK, IPOT_E_INVALID, IPOT_E_STATE, IPOT_E_NOMEM, IPOT_E_CUDA, IPOT_E_TIMEOUT, IPOT_E_BOUNDS, IPOT_E_LIMIT = 0, -1, -2, -3, -4, -5, -6, -7
 IPOT_NOALLOC_MAX_ROWS = 65536
 IPOT_BF16, IPOT_F32 = 0, 1
-IPOT_SCORER_AUTO, IPOT_SCORER_SIMT, IPOT_SCORER_TENSOR = 0, 1, 2
+IPOT_SCORER_AUTO, IPOT_SCORER_SIMT, IPOT_SCORER_TENSOR, IPOT_SCORER_WARP_MMA = 0, 1, 2, 3
 IPOT_ROPE_HALF, IPOT_ROPE_INTERLEAVED = 1, 2
 
 # every symbol include/ipot.h declares

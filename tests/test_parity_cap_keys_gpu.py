@@ -11,7 +11,7 @@ from parity import compare_cycle, from_dev_bits, gpu_cycle, make_pot, to_dev
 
 pytestmark = pytest.mark.gpu
 
-SCORERS = [ipot.IPOT_SCORER_SIMT, ipot.IPOT_SCORER_TENSOR]
+SCORERS = [ipot.IPOT_SCORER_SIMT, ipot.IPOT_SCORER_TENSOR, ipot.IPOT_SCORER_WARP_MMA]
 
 
 def with_cap_keys(cfg, cycle=0, scale=1.0):
@@ -60,6 +60,8 @@ def test_shapes_with_cap_keys(case, scorer):
     cfg = inputs.small_config(cfg_id=500 + case, **SHAPES[case])
     if scorer == ipot.IPOT_SCORER_TENSOR and not (cfg.dtype == "bf16" and cfg.d in (64, 128)):
         pytest.skip("the tensor scorer takes bf16 with d = 128 or 64")
+    if scorer == ipot.IPOT_SCORER_WARP_MMA and not (cfg.dtype == "bf16" and cfg.d % 16 == 0):
+        pytest.skip("the warp-level tensor-core scorer takes bf16 with d a multiple of 16")
     t = with_cap_keys(cfg)
     gpu = gpu_cycle(cfg, t, scorer)
     same, n = compare_cycle(cfg, t, gpu)

@@ -10,12 +10,21 @@ from parity import compare_cycle, from_dev_bits, gpu_cycle, make_pot, read_resul
 
 pytestmark = pytest.mark.gpu
 
-SCORERS = [ipot.IPOT_SCORER_SIMT, ipot.IPOT_SCORER_TENSOR]
+SCORERS = [ipot.IPOT_SCORER_SIMT, ipot.IPOT_SCORER_TENSOR, ipot.IPOT_SCORER_WARP_MMA]
 
 
 def tensor_scorer_applies(cfg, n=None):
     """The tcgen05 scorer takes bf16 with d = 128 or 64 (any pot size the library accepts)."""
     return cfg.dtype == "bf16" and cfg.d in (64, 128)
+
+
+def scorer_applies(cfg, scorer):
+    """fp32 FMAs: everything; tcgen05: see above; warp-level tensor cores: bf16 with d a multiple of 16."""
+    if scorer == ipot.IPOT_SCORER_TENSOR:
+        return tensor_scorer_applies(cfg)
+    if scorer == ipot.IPOT_SCORER_WARP_MMA:
+        return cfg.dtype == "bf16" and cfg.d % 16 == 0
+    return True
 
 
 def test_config1_tiny_f32_all_units():
@@ -46,6 +55,8 @@ SMALL = [
     dict(pot_size=2049, keep=1024, nuc_slots=512, cap_rows=16, Hq=8, Hkv=1, d=128, dtype="bf16", layers=2, batch=2),
     dict(pot_size=64, keep=63, nuc_slots=30, cap_rows=2, Hq=3, Hkv=3, d=256, dtype="f32", layers=3),
     dict(pot_size=1500, keep=700, nuc_slots=350, cap_rows=1, Hq=1, Hkv=1, d=128, dtype="bf16", batch=3),  # last-token rule
+    dict(pot_size=777, keep=300, nuc_slots=150, cap_rows=24, Hq=8, Hkv=2, d=256, dtype="bf16", layers=2),   # 256 channels
+    dict(pot_size=500, keep=250, nuc_slots=100, cap_rows=70, Hq=3, Hkv=1, d=96, dtype="bf16"),              # 96 channels, M = 210
 ]
 
 
@@ -53,9 +64,9 @@ SMALL = [
 @pytest.mark.parametrize("scorer", SCORERS)
 def test_small_random_shapes(case, scorer):
     cfg = inputs.small_config(cfg_id=200 + case, **SMALL[case])
-    if scorer == ipot.IPOT_SCORER_TENSOR and not tensor_scorer_applies(cfg):
+    if not scorer_applies(cfg, scorer):
         h = make_pot(cfg)
-        try:  # the tensor scorer must refuse, not fall back
+        try:  # a scorer that does not take the shape must refuse, not fall back
             t = inputs.make_cycle(cfg)
             ipot.ipot_set_scorer(h, scorer)
             ipot.ipot_append_chunk(h, to_dev(t["K"], cfg.dtype), to_dev(t["V"], cfg.dtype), cfg.pot_size)
