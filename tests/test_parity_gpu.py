@@ -341,3 +341,28 @@ def test_largest_pot_the_library_accepts(scorer):
     assert n == cfg.units and same == n
     rc = ipot.lib().ipot_create(32769, 8192, 1, 4, 1, 128, __import__("ctypes").byref(__import__("ctypes").c_void_p()))
     assert rc == ipot.IPOT_E_INVALID
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_seeded_random_configurations(seed):
+    """Shapes drawn from a seeded generator (pot fill, keep, NuC slots, CaP rows, heads, head dimension, dtype,
+    layers, streams): whatever scorer the library picks must agree with the checker, and so must every scorer
+    that accepts the shape."""
+    g = np.random.default_rng(9000 + seed)
+    dtype = "bf16" if g.random() < 0.7 else "f32"
+    d = int(g.choice([32, 48, 64, 96, 128, 160, 256]))
+    Hkv = int(g.choice([1, 2, 3]))
+    G = int(g.choice([1, 2, 4, 5]))
+    pot = int(g.integers(70, 1400))
+    n = int(g.integers(max(2, pot // 2), pot + 1))
+    keep = int(g.integers(1, n))
+    T = int(g.integers(0, keep + 1))
+    cfg = inputs.small_config(cfg_id=900 + seed, pot_size=pot, keep=keep, nuc_slots=T, cap_rows=int(g.integers(1, 40)),
+                              Hq=Hkv * G, Hkv=Hkv, d=d, dtype=dtype, layers=int(g.integers(1, 3)), batch=int(g.integers(1, 3)))
+    t = inputs.make_cycle(cfg)
+    for scorer in [ipot.IPOT_SCORER_AUTO] + SCORERS:
+        if scorer != ipot.IPOT_SCORER_AUTO and not scorer_applies(cfg, scorer):
+            continue
+        gpu = gpu_cycle(cfg, t, scorer, n=n)
+        same, cnt = compare_cycle(cfg, t, gpu, n=n)
+        assert cnt == cfg.units and same >= cnt - 1, (seed, scorer)
