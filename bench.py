@@ -35,6 +35,7 @@ NOVELTY_WORKLOADS = {"nuc32k": (32000, 2048), "nuc128k": (128256, 2048)}
 # generation over a full pot alone: one new token's attention over all layers' units, configs[cfg - 1] shape
 DECODE_WORKLOADS = {"decode3": 3, "decode4": 4, "decode5": 5}
 RING = 4  # distinct chunks / query sets cycled through
+PREHEAT_S = 0.5  # untimed running before the warm-up steps, see main()
 
 
 def peaks():
@@ -546,14 +547,27 @@ def main():
         rate, ms_step = whole_job_rate(e0.elapsed_time(e1), steps, world, "cuda")
         return rate, ms_step, ipot.ipot_launch_count(h) - l0, clocks
 
-    # device-resident inputs: the headline value, with per-kernel events over the same timed region
+    # untimed pre-heat: the first few hundred milliseconds after idle run at lower memory throughput (the compaction
+    # kernel takes 105 us averaged over the first 0.1 s of steps, 91 us over 0.3 s, 82 us afterwards)
+    t_end = time.perf_counter() + PREHEAT_S
+    i = 0
+    while time.perf_counter() < t_end:
+        for _ in range(50):
+            step_dev(i)
+            i += 1
+        torch.cuda.synchronize()
+    # device-resident inputs: the headline value over exactly K steps, no instrumentation inside the region
+    sampler = ClockSampler(local)
+    value, ms_step, launches, clocks = timed(step_dev, args.steps, args.warmup, sampler)
+    assert ipot.ipot_sync_status(h) == 0, "device status is not clean"
+    # the same K steps once more with the library's per-kernel CUDA events (they serialise the kernel boundaries,
+    # which costs a few microseconds per step: reported beside the headline, not as it)
     ipot.ipot_set_profiling(h, 1)
-    for i in range(args.warmup):
+    for i in range(3):
         step_dev(i)
     torch.cuda.synchronize()
     ipot.ipot_kernel_ms(h)  # drop the warm-up cycles from the per-kernel means
-    sampler = ClockSampler(local)
-    value, ms_step, launches, clocks = timed(step_dev, args.steps, 0, sampler)
+    _, ms_step_events, _, _ = timed(step_dev, args.steps, 0)
     kms, kcycles, scorer_used = ipot.ipot_kernel_ms(h)
     ipot.ipot_set_profiling(h, 0)
     assert ipot.ipot_sync_status(h) == 0, "device status is not clean"
@@ -597,9 +611,10 @@ def main():
         "metric": "ccd_cycles_per_s", "value": value, "unit": "cycles/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
-        "config": config_dict(cfg, n_new, N, args.cap_keys, getattr(args, "rope", False)),
+        "config": dict(config_dict(cfg, n_new, N, args.cap_keys, getattr(args, "rope", False)), preheat_s=PREHEAT_S),
         "pot_tokens_per_s": value * N * cfg.batch,
         "layer_cycles_per_s": value * cfg.layers,
+        "ms_per_step_with_kernel_events": ms_step_events,
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": "cycles/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "steps": e2e_steps},
