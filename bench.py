@@ -449,6 +449,9 @@ def main():
     ap.add_argument("--rope", action="store_true",
                     help="context-reset rotary mode: unrotated keys in the pot, the row movers keep a rotated copy")
     ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (profiling small cases)")
+    ap.add_argument("--append", default="deferred", choices=["deferred", "eager"],
+                    help="deferred: the chunk stays in the caller's buffers, the scorer reads its keys there and the "
+                         "compaction fetches the surviving rows (ipot_set_deferred_append); eager: copied at append")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.workload in NOVELTY_WORKLOADS:
@@ -502,6 +505,7 @@ def main():
         ipot.ipot_enable_rope(h, rope_tables[0], rope_tables[1], ipot.IPOT_ROPE_HALF)
     stream = torch.cuda.current_stream()
     ipot.ipot_set_stream(h, stream.cuda_stream)
+    ipot.ipot_set_deferred_append(h, args.append == "deferred")
     ipot.ipot_append_chunk(h, K0d, V0d, cfg.keep)
 
     small_l2 = cfg.units * N * cfg.d * cfg.elem_bytes * 2 <= 126e6
@@ -571,6 +575,11 @@ def main():
     kms, kcycles, scorer_used = ipot.ipot_kernel_ms(h)
     ipot.ipot_set_profiling(h, 0)
     assert ipot.ipot_sync_status(h) == 0, "device status is not clean"
+    # the same K steps with the other append mode, for comparison
+    ipot.ipot_set_deferred_append(h, args.append != "deferred")
+    _, ms_step_other, _, _ = timed(step_dev, args.steps, 3)
+    ipot.ipot_set_deferred_append(h, args.append == "deferred")
+    assert ipot.ipot_sync_status(h) == 0, "device status is not clean"
 
     # end to end: host (pinned) buffers in, index lists out, copies inside the timed region
     e2e_steps = max(3, min(args.steps, 50))
@@ -611,10 +620,14 @@ def main():
         "metric": "ccd_cycles_per_s", "value": value, "unit": "cycles/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
-        "config": dict(config_dict(cfg, n_new, N, args.cap_keys, getattr(args, "rope", False)), preheat_s=PREHEAT_S),
+        "config": dict(config_dict(cfg, n_new, N, args.cap_keys, getattr(args, "rope", False)), preheat_s=PREHEAT_S,
+                       append=("deferred: the chunk stays in the caller's device buffers, the scorer reads its keys there, "
+                               "the compaction copies the surviving rows into the pot" if args.append == "deferred"
+                               else "eager: all rows copied into the pot by the append call")),
         "pot_tokens_per_s": value * N * cfg.batch,
         "layer_cycles_per_s": value * cfg.layers,
         "ms_per_step_with_kernel_events": ms_step_events,
+        ("ms_per_step_eager_append" if args.append == "deferred" else "ms_per_step_deferred_append"): ms_step_other,
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": "cycles/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "steps": e2e_steps},

@@ -120,6 +120,23 @@ int ipot_reset(ipot_t *pot);
  */
 int ipot_append_chunk(ipot_t *pot, const void *K, const void *V, int n_tokens);
 
+/*
+ * Deferred append (off by default).  While it is on, ipot_append_chunk() copies nothing: it notes the caller's
+ * buffers, and the rows are taken from there when they are needed -
+ *   - the tensor-core scorer reads the new keys in place (when the fill before the append is a multiple of 256;
+ *     otherwise, and for every other scorer, the keys are copied into the pot first);
+ *   - the compaction of the next cycle (Appendix B, "KV-cache compression") fetches the surviving rows from the
+ *     chunk, so rows that the cycle drops are never copied and survivors move once instead of twice;
+ *   - every other call that reads or exposes the pot's rows (ipot_view, ipot_decode_attention, a further append,
+ *     ipot_append_chunk_host, ipot_set_stream, ipot_sync_status, turning the mode off) first queues the plain copy.
+ * In rotary mode only the values are deferred (the scorers read the rotated copy, which is written at append).
+ * The pot's contents after any of these calls are the same as without the mode.  What changes is the lifetime of
+ * the chunk buffers: they must stay alive and unchanged until the next ipot_score_and_compress*() has run on the
+ * stream or ipot_sync_status() has returned - synchronising the stream right after the append is not enough.
+ * Errors: INVALID (NULL pot), CUDA.
+ */
+int ipot_set_deferred_append(ipot_t *pot, int on);
+
 /* Same with HOST buffers (pinned memory makes the copy asynchronous): the
  * rows go straight from host memory into the pot with strided copies. */
 int ipot_append_chunk_host(ipot_t *pot, const void *K_host, const void *V_host, int n_tokens);

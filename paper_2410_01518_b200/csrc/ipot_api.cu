@@ -31,6 +31,12 @@ struct ipot {
     int G, units, elem_bytes, row_bytes;
     int compact_slices, rope_slices;
     cudaStream_t stream;
+    // Deferred append (ipot_set_deferred_append): the newest chunk's rows (slots pend_first .. len - 1) still lie in
+    // the caller's buffers; the tensor-core scorer reads its keys there and the compaction fetches the survivors
+    // from there, so rows that the cycle drops are never copied.  NULL = those rows are in the pot.
+    int deferred;
+    const void *pend_K, *pend_V;
+    int pend_n, pend_first;
     // device memory (library-owned)
     void *K, *V;
     // CR-RoPE (ipot_enable_rope): K then holds the keys without rotary embedding, Krot the copy rotated at the slot
@@ -115,6 +121,38 @@ void free_all(ipot *p)
     }
 }
 
+// Copies the rows of a deferred append that are still in the caller's buffers into the pot (keys, values or both).
+int materialise(ipot *p, bool keys, bool values)
+{
+    const void *k = keys ? p->pend_K : nullptr, *v = values ? p->pend_V : nullptr;
+    if (!k && !v) return IPOT_OK;
+    const size_t row_vecs = p->row_bytes / 16, n_vecs = (size_t)p->pend_n * row_vecs;
+    int pieces = (int)((n_vecs + (size_t)kMoveThreads * kMoveVecs - 1) / ((size_t)kMoveThreads * kMoveVecs));
+    if (pieces < 1) pieces = 1;
+    dim3 grid(pieces, p->units, (k && v) ? 2 : 1);
+    if (k && v)
+        append_kernel<<<grid, kMoveThreads, 0, p->stream>>>((const uint4 *)k, (const uint4 *)v, (uint4 *)p->K, (uint4 *)p->V, n_vecs,
+                                                           (size_t)p->cfg.pot_size * row_vecs, (size_t)p->pend_first * row_vecs);
+    else
+        append_kernel<<<grid, kMoveThreads, 0, p->stream>>>((const uint4 *)(k ? k : v), nullptr, (uint4 *)(k ? p->K : p->V), nullptr, n_vecs,
+                                                           (size_t)p->cfg.pot_size * row_vecs, (size_t)p->pend_first * row_vecs);
+    p->launches += 1;
+    IPOT_CUDA(cudaGetLastError());
+    if (k) p->pend_K = nullptr;
+    if (v) p->pend_V = nullptr;
+    return IPOT_OK;
+}
+
+PendingRows pending_rows(const ipot *p)
+{
+    PendingRows r;
+    r.K = (const uint4 *)p->pend_K;
+    r.V = (const uint4 *)p->pend_V;
+    r.unit_vecs = (size_t)p->pend_n * (p->row_bytes / 16);
+    r.first = p->pend_first;
+    return r;
+}
+
 // Row statistics over the CaP's own keys (causal): what Appendix B's listing adds to every row's denominator.
 int launch_cap_self(ipot *p, const void *Q, const void *Kc, int M, int P)
 {
@@ -190,6 +228,13 @@ int run_scoring(ipot *p, const void *Q, const void *Kc, int cap_rows, const floa
     if (scorer == IPOT_SCORER_TENSOR && !tc_ok) return IPOT_E_INVALID;
     if (scorer == IPOT_SCORER_WARP_MMA && !mma_ok) return IPOT_E_INVALID;
     if (scorer == IPOT_SCORER_AUTO) scorer = tc_ok ? IPOT_SCORER_TENSOR : mma_ok ? IPOT_SCORER_WARP_MMA : IPOT_SCORER_SIMT;
+    // keys of a deferred append: the tensor-core scorer reads whole slabs of them where they are, anything else
+    // wants them in the pot
+    const bool keys_in_chunk = p->pend_K && scorer == IPOT_SCORER_TENSOR && p->pend_first % kTcSlab == 0;
+    if (p->pend_K && !keys_in_chunk) {
+        int mrc = materialise(p, true, false);
+        if (mrc != IPOT_OK) return mrc;
+    }
 
     cudaEvent_t *ev = (p->profiling && p->ev_used < kProfSlots) ? p->ev[p->ev_used] : nullptr;
     if (ev) IPOT_CUDA(cudaEventRecord(ev[0], p->stream));
@@ -209,7 +254,7 @@ int run_scoring(ipot *p, const void *Q, const void *Kc, int cap_rows, const floa
     if (scorer == IPOT_SCORER_TENSOR) {
         int n_launch = 0;
         rc = tc_launch(p->tc, p->cfg, Q, score_keys(p), cap_stats, p->scores, (size_t)p->units * p->cfg.pot_size, N, M, p->units, p->status,
-                       p->stream, parts, &n_launch);
+                       p->stream, parts, &n_launch, keys_in_chunk ? p->pend_K : nullptr, keys_in_chunk ? p->pend_first : 0);
         p->launches += n_launch;
     } else if (scorer == IPOT_SCORER_WARP_MMA) {
         rc = launch_warp_mma(p, Q, cap_stats, M, N);
@@ -242,7 +287,7 @@ void launch_compact_rope_t(ipot *p, int keep, int N, int row_vecs, size_t unit_v
     auto kern = p->rope == IPOT_ROPE_INTERLEAVED ? compact_rope_kernel<T, true> : compact_rope_kernel<T, false>;
     kern<<<grid, kMoveThreads, 0, p->stream>>>((uint4 *)p->K, (uint4 *)p->Krot, (const T *)p->rope_cos, (const T *)p->rope_sin, p->idx,
                                                keep, N, row_vecs, ks, row_vecs / 2 / ks, unit_vecs, p->status, (uint4 *)p->V, vs,
-                                               row_vecs / vs);
+                                               row_vecs / vs, pending_rows(p));
 }
 
 void launch_compact_rope(ipot *p, int keep, int N, int row_vecs, size_t unit_vecs)
@@ -315,13 +360,14 @@ int run_cycle(ipot *p, const void *Q, const void *Kc, int cap_rows, const float 
     if (!p->rope) {
         dim3 grid(slices, p->units, 2);
         compact_kernel<<<grid, kMoveThreads, 0, p->stream>>>((uint4 *)p->K, (uint4 *)p->V, p->idx, keep, N, row_vecs,
-                                                            row_vecs / slices, unit_vecs, p->status);
+                                                            row_vecs / slices, unit_vecs, p->status, pending_rows(p));
         p->launches += 1;
     } else {
         launch_compact_rope(p, keep, N, row_vecs, unit_vecs);
         p->launches += 1;
     }
     IPOT_CUDA(cudaGetLastError());
+    p->pend_K = p->pend_V = nullptr;  // the survivors are in the pot, the rest of the chunk is dropped
     if (ev) {
         IPOT_CUDA(cudaEventRecord(ev[4], p->stream));
         p->ev_used += 1;
@@ -517,6 +563,8 @@ int ipot_destroy(ipot_t *p)
 int ipot_set_stream(ipot_t *p, void *s)
 {
     if (!p) return IPOT_E_INVALID;
+    int rc = materialise(p, true, true);  // queued on the stream that is being left
+    if (rc != IPOT_OK) return rc;
     p->stream = (cudaStream_t)s;
     return IPOT_OK;
 }
@@ -535,10 +583,22 @@ int ipot_set_scorer(ipot_t *p, int scorer)
     return IPOT_OK;
 }
 
+int ipot_set_deferred_append(ipot_t *p, int on)
+{
+    if (!p) return IPOT_E_INVALID;
+    if (!on) {
+        int rc = materialise(p, true, true);
+        if (rc != IPOT_OK) return rc;
+    }
+    p->deferred = on ? 1 : 0;
+    return IPOT_OK;
+}
+
 int ipot_reset(ipot_t *p)
 {
     if (!p) return IPOT_E_INVALID;
     p->len = 0;
+    p->pend_K = p->pend_V = nullptr;
     p->tc.last_items = 0;  // the tensor scorer clears its statistics array before its next launch
     return IPOT_OK;
 }
@@ -551,6 +611,22 @@ int ipot_append_chunk(ipot_t *p, const void *K, const void *V, int n)
     const size_t n_vecs = (size_t)n * row_vecs;
     int pieces = (int)((n_vecs + (size_t)kMoveThreads * kMoveVecs - 1) / ((size_t)kMoveThreads * kMoveVecs));
     if (pieces < 1) pieces = 1;
+    int rc = materialise(p, true, true);  // at most one chunk is kept outside the pot
+    if (rc != IPOT_OK) return rc;
+    if (p->deferred) {
+        p->pend_first = p->len;
+        p->pend_n = n;
+        p->pend_V = V;
+        if (!p->rope) {
+            p->pend_K = K;
+        } else {  // the rotated copy is what the scorers read: the keys go into the pot now, the values wait
+            launch_append_rope(p, K, n_vecs, nullptr, n);
+            p->launches += 1;
+            IPOT_CUDA(cudaGetLastError());
+        }
+        p->len += n;
+        return IPOT_OK;
+    }
     if (!p->rope) {
         dim3 grid(pieces, p->units, 2);
         append_kernel<<<grid, kMoveThreads, 0, p->stream>>>((const uint4 *)K, (const uint4 *)V, (uint4 *)p->K, (uint4 *)p->V,
@@ -568,6 +644,8 @@ int ipot_append_chunk_host(ipot_t *p, const void *K, const void *V, int n)
 {
     if (!p || !K || !V || n <= 0) return IPOT_E_INVALID;
     if (p->len + n > p->cfg.pot_size) return IPOT_E_STATE;
+    int rc = materialise(p, true, true);
+    if (rc != IPOT_OK) return rc;
     const size_t width = (size_t)n * p->row_bytes, dpitch = (size_t)p->cfg.pot_size * p->row_bytes;
     char *dK = (char *)p->K + (size_t)p->len * p->row_bytes, *dV = (char *)p->V + (size_t)p->len * p->row_bytes;
     IPOT_CUDA(cudaMemcpy2DAsync(dK, dpitch, K, width, width, p->units, cudaMemcpyHostToDevice, p->stream));
@@ -698,6 +776,8 @@ int ipot_decode_attention(ipot_t *p, const void *q, float *out, float *lse)
     if (p->row_bytes % 16 || (lpk != 4 && lpk != 8 && lpk != 16 && lpk != 32)) return IPOT_E_INVALID;
     if (p->G > 8) return IPOT_E_INVALID;
     if (p->len < 1) return IPOT_E_STATE;
+    int rc = materialise(p, true, true);
+    if (rc != IPOT_OK) return rc;
     if (p->cfg.dtype == IPOT_BF16 && p->scorer != IPOT_SCORER_SIMT && (p->cfg.d == 64 || p->cfg.d == 128))
         return p->cfg.d == 64 ? launch_decode_mma<64>(p, q, out, lse) : launch_decode_mma<128>(p, q, out, lse);
     if (p->G != 1 && p->G != 2 && p->G != 4 && p->G != 8) return IPOT_E_INVALID;
@@ -735,6 +815,8 @@ int ipot_view_rope(ipot_t *p, void **K_rot)
 int ipot_view(ipot_t *p, void **K, void **V, int *len)
 {
     if (!p) return IPOT_E_INVALID;
+    int rc = materialise(p, true, true);
+    if (rc != IPOT_OK) return rc;
     if (K) *K = p->K;
     if (V) *V = p->V;
     if (len) *len = p->len;
@@ -759,6 +841,8 @@ int ipot_last_scores(ipot_t *p, const float **u, int *len_before)
 int ipot_sync_status(ipot_t *p)
 {
     if (!p) return IPOT_E_INVALID;
+    int rc = materialise(p, true, true);  // after this call the caller's chunk buffers are free again
+    if (rc != IPOT_OK) return rc;
     IPOT_CUDA(cudaStreamSynchronize(p->stream));
     int st = 0;
     IPOT_CUDA(cudaMemcpy(&st, p->status, sizeof(int), cudaMemcpyDeviceToHost));

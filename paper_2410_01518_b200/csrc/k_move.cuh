@@ -26,7 +26,8 @@ __device__ __forceinline__ void append_body(const uint4 *__restrict__ src, uint4
     for (; v < n_vecs; v += stride) dst[v] = __ldg(src + v);
 }
 
-// grid (pieces, units, 2): tensor z of unit y; src is [units][n_vecs], dst is the pot.
+// grid (pieces, units, 1 or 2): tensor z of unit y (z = 0 alone: the first pair of pointers); src is [units][n_vecs],
+// dst is the pot.
 __global__ void __launch_bounds__(kMoveThreads)
 append_kernel(const uint4 *__restrict__ srcK, const uint4 *__restrict__ srcV, uint4 *__restrict__ potK,
               uint4 *__restrict__ potV, size_t n_vecs, size_t unit_vecs, size_t first_vec)
@@ -44,9 +45,14 @@ append_kernel(const uint4 *__restrict__ srcK, const uint4 *__restrict__ srcV, ui
 // writes land in rows below the next chunk's first row, and every later source
 // row lies at or above it, so nothing that is still needed is overwritten.
 // Rows with idx[r] == r are left alone.
-// base: the block's first vector of row 0 (its byte-column slice of one tensor of one unit)
+// base: the block's first vector of row 0 (its byte-column slice of one tensor of one unit).
+// Rows from alt_first on may still lie outside the pot, in the caller's chunk of a deferred append: alt is then the
+// block's first vector of the chunk's row 0 (same byte columns; slot alt_first), else alt_first = INT_MAX.  Such
+// rows are fetched from there, also when they keep their slot number, so after the gather the pot holds every
+// survivor and nothing else of the chunk was ever copied.
 __device__ __forceinline__ void compact_body(uint4 *__restrict__ base, const int32_t *__restrict__ ix, int keep, int N,
-                                             int row_vecs, int slice_vecs, int *status)
+                                             int row_vecs, int slice_vecs, int *status, const uint4 *__restrict__ alt = nullptr,
+                                             int alt_first = 0x7fffffff)
 {
     const int rows_per_pass = kMoveThreads / slice_vecs;  // rows covered by one vector per thread
     const int chunk_rows = rows_per_pass * kMoveVecs;
@@ -61,12 +67,14 @@ __device__ __forceinline__ void compact_body(uint4 *__restrict__ base, const int
             if (r < keep && my_row < rows_per_pass) {
                 const int s = ix[r];
                 if (s < r || s >= N) set_status(status, kStatusBounds);
-                else if (s != r) src[i] = s;
+                else if (s != r || s >= alt_first) src[i] = s;
             }
         }
 #pragma unroll
         for (int i = 0; i < kMoveVecs; ++i)
-            if (src[i] >= 0) t[i] = base[(size_t)src[i] * row_vecs + my_vec];
+            if (src[i] >= 0)
+                t[i] = src[i] >= alt_first ? __ldg(alt + (size_t)(src[i] - alt_first) * row_vecs + my_vec)
+                                           : base[(size_t)src[i] * row_vecs + my_vec];
         __syncthreads();
 #pragma unroll
         for (int i = 0; i < kMoveVecs; ++i) {
@@ -76,12 +84,22 @@ __device__ __forceinline__ void compact_body(uint4 *__restrict__ base, const int
     }
 }
 
+// A deferred append's chunk: rows of slot numbers first, first + 1, ... of every unit, still in the caller's buffers
+// ([units][rows][row_vecs]); K or V is NULL where the pot already holds those rows.
+struct PendingRows {
+    const uint4 *K, *V;
+    size_t unit_vecs;  // rows * row_vecs
+    int first;
+};
+
 __global__ void __launch_bounds__(kMoveThreads)
 compact_kernel(uint4 *__restrict__ potK, uint4 *__restrict__ potV, const int32_t *__restrict__ idx,
-               int keep, int N, int row_vecs, int slice_vecs, size_t unit_vecs, int *status)
+               int keep, int N, int row_vecs, int slice_vecs, size_t unit_vecs, int *status, PendingRows pend)
 {
     uint4 *base = (blockIdx.z ? potV : potK) + (size_t)blockIdx.y * unit_vecs + (size_t)blockIdx.x * slice_vecs;
-    compact_body(base, idx + (size_t)blockIdx.y * keep, keep, N, row_vecs, slice_vecs, status);
+    const uint4 *alt = blockIdx.z ? pend.V : pend.K;
+    if (alt) alt += (size_t)blockIdx.y * pend.unit_vecs + (size_t)blockIdx.x * slice_vecs;
+    compact_body(base, idx + (size_t)blockIdx.y * keep, keep, N, row_vecs, slice_vecs, status, alt, alt ? pend.first : 0x7fffffff);
 }
 
 }  // namespace ipotk

@@ -195,17 +195,20 @@ append_rope_kernel(const uint4 *__restrict__ src, size_t src_unit_vecs, uint4 *p
 // owns the vector pairs (g, g + row_vecs / 2) with g in [slice * slice_vecs, (slice + 1) * slice_vecs) of every row
 // of one unit; the walk over the rows is compact_kernel's (ascending chunks, read - barrier - write), which is
 // safe in place because idx[r] >= r.  The rotated copy is only written, never read.
-// z = 1 (if launched): the value rows, compact_kernel's walk with its own slicing (v_slices slices of v_slice_vecs).
+// z = 1 (if launched): the value rows, compact_kernel's walk with its own slicing (v_slices slices of v_slice_vecs);
+// pend.V names the value rows of a deferred append, if any (pend.K is not used: the keys are in the pot).
 template <typename T, bool kInterleaved>
 __global__ void __launch_bounds__(kMoveThreads)
 compact_rope_kernel(uint4 *potK, uint4 *__restrict__ potKrot, const T *__restrict__ cos_t, const T *__restrict__ sin_t,
                     const int32_t *__restrict__ idx, int keep, int N, int row_vecs, int k_slices, int slice_vecs, size_t unit_vecs,
-                    int *status, uint4 *potV, int v_slices, int v_slice_vecs)
+                    int *status, uint4 *potV, int v_slices, int v_slice_vecs, PendingRows pend)
 {
     if (blockIdx.z == 1) {
-        if ((int)blockIdx.x < v_slices)
+        if ((int)blockIdx.x < v_slices) {
+            const uint4 *alt = pend.V ? pend.V + (size_t)blockIdx.y * pend.unit_vecs + (size_t)blockIdx.x * v_slice_vecs : nullptr;
             compact_body(potV + (size_t)blockIdx.y * unit_vecs + (size_t)blockIdx.x * v_slice_vecs, idx + (size_t)blockIdx.y * keep,
-                         keep, N, row_vecs, v_slice_vecs, status);
+                         keep, N, row_vecs, v_slice_vecs, status, alt, alt ? pend.first : 0x7fffffff);
+        }
         return;
     }
     if ((int)blockIdx.x >= k_slices) return;

@@ -65,7 +65,9 @@ constexpr uint32_t kTcOffColpart = 2 * kTcStageBytes;                      // [2
 constexpr uint32_t kTcOffTstat = kTcOffColpart + 2 * 4 * kTcSlab * 4;          // [2 buffers][8 chunks][128] float2
 constexpr uint32_t kTcOffFbuf = kTcOffTstat + 2 * 8 * kTcRows * 8;         // [2 buffers][8 chunks][128] float
 constexpr uint32_t kTcOffBar = kTcOffFbuf + 2 * 8 * kTcRows * 4;
-constexpr uint32_t kTcSmemBytes = kTcOffBar + 256 + 1024;                  // + alignment slack
+constexpr uint32_t kTcOffTmemSlot = kTcOffBar + 128;                       // the allocated TMEM base address
+constexpr uint32_t kTcOffAbort = kTcOffBar + 132;                          // set once a wait of the CTA has run out
+constexpr uint32_t kTcSmemBytes = kTcOffBar + 256;                         // no static shared memory: the base is 1024-aligned
 
 // barriers: per stage Full, Empty, EReady, FReady; per (buffer, half) SFull, TEmpty at index 2 * buffer + half
 enum { kBarFull = 0, kBarEmpty = 2, kBarEReady = 4, kBarFReady = 6, kBarSFull = 8, kBarTEmpty = 12, kBarCount = 16 };
@@ -79,6 +81,8 @@ struct TcParams {
     int *status;
     int N, M, mtiles, slabs, tasks;
     int dhalves;          // d / 64: 64-channel halves of a tile (1 or 2)
+    int new_slab0;        // slabs from this one on are read through the second key map (the chunk of a deferred
+                          // append, row 0 = key 256 * new_slab0); INT_MAX if all keys are in the pot
     float scale_log2e;
 };
 
@@ -200,9 +204,15 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 // Named barrier of the four epilogue warps (one per TMEM lane quarter) that own the same columns.
+// (Barrier numbers are immediates so that the kernel claims five of the SM's barriers, not all sixteen.)
 __device__ __forceinline__ void column_group_sync(int cq)
 {
-    asm volatile("bar.sync %0, 128;" ::"r"(1 + cq) : "memory");
+    switch (cq) {
+    case 0: asm volatile("bar.sync 1, 128;" ::: "memory"); break;
+    case 1: asm volatile("bar.sync 2, 128;" ::: "memory"); break;
+    case 2: asm volatile("bar.sync 3, 128;" ::: "memory"); break;
+    default: asm volatile("bar.sync 4, 128;" ::: "memory"); break;
+    }
 }
 // The slab statistics are exchanged between CTAs with single 8-byte relaxed accesses at gpu scope:
 // one store publishes (max, marked sum) together, and a reader sees either the old or the new pair.
@@ -333,14 +343,18 @@ constexpr uint32_t kTcIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) 
 
 // ------------------------------------------------------------------ the kernel
 __global__ void __launch_bounds__(kTcThreads, 1)
-cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK, TcParams prm)
+cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
+                    const __grid_constant__ CUtensorMap mapKnew, TcParams prm)
 {
-    extern __shared__ uint8_t tc_smem_raw[];
-    __shared__ uint32_t tmem_base_slot;
-    __shared__ int abort_flag;
-
-    const uint32_t base = (smem_u32(tc_smem_raw) + 1023u) & ~1023u;
-    uint8_t *gbase = tc_smem_raw + (base - smem_u32(tc_smem_raw));
+    extern __shared__ __align__(1024) uint8_t tc_smem_raw[];
+    const uint32_t base = smem_u32(tc_smem_raw);
+    if (base & 1023u) {  // the swizzled tiles need this alignment; nothing has been started yet
+        if (threadIdx.x == 0) set_status(prm.status, kStatusBounds);
+        return;
+    }
+    uint8_t *gbase = tc_smem_raw;
+    uint32_t &tmem_base_slot = *reinterpret_cast<uint32_t *>(gbase + kTcOffTmemSlot);
+    int &abort_flag = *reinterpret_cast<int *>(gbase + kTcOffAbort);
     const uint32_t bar0 = base + kTcOffBar;
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -381,11 +395,14 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                 mbar_wait(bar(kBarEmpty + b), ph ^ 1, ab, prm.status);
                 mbar_expect_tx(bar(kBarFull + b), (uint32_t)prm.dhalves * (kTcStageBytes / 2));
                 const uint32_t q = base + kTcOffStage + b * kTcStageBytes, kk = q + kTcQBytes;
+                const bool fresh_rows = slab >= prm.new_slab0;
+                const CUtensorMap *mk = fresh_rows ? &mapKnew : &mapK;
+                const int krow = (fresh_rows ? slab - prm.new_slab0 : slab) * kTcSlab;
                 tma_load_3d(q, &mapQ, 0, mt * kTcRows, unit, bar(kBarFull + b));
-                tma_load_3d(kk, &mapK, 0, slab * kTcSlab, unit, bar(kBarFull + b));
+                tma_load_3d(kk, mk, 0, krow, unit, bar(kBarFull + b));
                 if (prm.dhalves == 2) {
                     tma_load_3d(q + kTcQBytes / 2, &mapQ, 64, mt * kTcRows, unit, bar(kBarFull + b));
-                    tma_load_3d(kk + kTcKBytes / 2, &mapK, 64, slab * kTcSlab, unit, bar(kBarFull + b));
+                    tma_load_3d(kk + kTcKBytes / 2, mk, 64, krow, unit, bar(kBarFull + b));
                 }
             }
         }
@@ -656,20 +673,32 @@ inline int tc_encode_rows(TcPlan &plan, CUtensorMap *map, const void *ptr, int d
 }
 
 // scores: partial array p (query rows 128 p ...) is written at scores + p * part_stride, unit stride N.
+// Knew (may be NULL): the keys from slot new_first on are not in the pot yet but in this [units][N - new_first][d]
+// array (the chunk of a deferred append); new_first must be a multiple of the slab size.
 inline int tc_launch(TcPlan &plan, const ipot_config_t &cfg, const void *Q, const void *K, const float2 *cap_stats, float *scores,
-                     size_t part_stride, int N, int M, int units, int *status, cudaStream_t stream, int *parts, int *n_launch)
+                     size_t part_stride, int N, int M, int units, int *status, cudaStream_t stream, int *parts, int *n_launch,
+                     const void *Knew = nullptr, int new_first = 0)
 {
     if (!tc_applicable(plan, cfg, N, M)) return IPOT_E_INVALID;
+    if (Knew && (new_first % kTcSlab != 0 || new_first >= N)) return IPOT_E_INVALID;
     const int mtiles = (M + kTcRows - 1) / kTcRows;
-    CUtensorMap mapQ, mapK;
+    CUtensorMap mapQ, mapK, mapKnew;
     if (tc_encode_rows(plan, &mapQ, Q, cfg.d, M, units, (size_t)M, kTcRows) != IPOT_OK) return IPOT_E_CUDA;
-    if (tc_encode_rows(plan, &mapK, K, cfg.d, N, units, (size_t)cfg.pot_size, kTcSlab) != IPOT_OK) return IPOT_E_CUDA;
+    if (Knew && new_first == 0) {  // every key is in the chunk
+        if (tc_encode_rows(plan, &mapK, Knew, cfg.d, N, units, (size_t)N, kTcSlab) != IPOT_OK) return IPOT_E_CUDA;
+        Knew = nullptr;
+    } else if (tc_encode_rows(plan, &mapK, K, cfg.d, Knew ? new_first : N, units, (size_t)cfg.pot_size, kTcSlab) != IPOT_OK) {
+        return IPOT_E_CUDA;
+    }
+    if (!Knew) mapKnew = mapK;
+    else if (tc_encode_rows(plan, &mapKnew, Knew, cfg.d, N - new_first, units, (size_t)(N - new_first), kTcSlab) != IPOT_OK) return IPOT_E_CUDA;
     TcParams prm;
     prm.scores = scores; prm.part_stride = part_stride; prm.stats = plan.stats; prm.cap_stats = cap_stats; prm.status = status;
     prm.N = N; prm.M = M; prm.mtiles = mtiles; prm.slabs = (N + kTcSlab - 1) / kTcSlab;
     const int items = units * mtiles;
     prm.tasks = items * prm.slabs;
     prm.dhalves = cfg.d / 64;
+    prm.new_slab0 = Knew ? new_first / kTcSlab : 0x7fffffff;
     prm.scale_log2e = (float)(1.4426950408889634 / sqrt((double)cfg.d));
     if (items != plan.last_items || prm.slabs != plan.last_slabs) {
         if (cudaMemsetAsync(plan.stats, 0, (size_t)items * prm.slabs * kTcRows * sizeof(float2), stream) != cudaSuccess) {
@@ -690,7 +719,7 @@ inline int tc_launch(TcPlan &plan, const ipot_config_t &cfg, const void *Q, cons
     at[0].id = cudaLaunchAttributeCooperative;  // all CTAs resident: they wait on each other's statistics
     at[0].val.cooperative = 1;
     lc.attrs = at; lc.numAttrs = 1;
-    if (cudaLaunchKernelEx(&lc, cap_score_tc_kernel, mapQ, mapK, prm) != cudaSuccess) {
+    if (cudaLaunchKernelEx(&lc, cap_score_tc_kernel, mapQ, mapK, mapKnew, prm) != cudaSuccess) {
         cudaGetLastError();
         return IPOT_E_CUDA;
     }

@@ -25,7 +25,7 @@ IPOT_ROPE_HALF, IPOT_ROPE_INTERLEAVED = 1, 2
 # every symbol include/ipot.h declares
 SYMBOLS = [
     "ipot_create", "ipot_create_ex", "ipot_destroy", "ipot_set_stream", "ipot_set_nuc_slots",
-    "ipot_set_scorer", "ipot_reset", "ipot_append_chunk", "ipot_append_chunk_host",
+    "ipot_set_scorer", "ipot_set_deferred_append", "ipot_reset", "ipot_append_chunk", "ipot_append_chunk_host",
     "ipot_score_and_compress", "ipot_score_and_compress_host", "ipot_score_only", "ipot_view",
     "ipot_last_indices", "ipot_last_scores", "ipot_sync_status", "ipot_set_profiling",
     "ipot_kernel_ms", "ipot_launch_count", "ipot_strerror", "ipot_cap_scores_noalloc",
@@ -69,6 +69,7 @@ def lib() -> C.CDLL:
         L.ipot_set_stream.argtypes = [vp, vp]
         L.ipot_set_nuc_slots.argtypes = [vp, ip]
         L.ipot_set_scorer.argtypes = [vp, ip]
+        L.ipot_set_deferred_append.argtypes = [vp, ip]
         L.ipot_reset.argtypes = [vp]
         L.ipot_append_chunk.argtypes = [vp, vp, vp, ip]
         L.ipot_append_chunk_host.argtypes = [vp, vp, vp, ip]
@@ -147,6 +148,10 @@ def ipot_set_nuc_slots(h, T) -> None:
 
 def ipot_set_scorer(h, scorer) -> None:
     _check(lib().ipot_set_scorer(h, scorer), "ipot_set_scorer")
+
+
+def ipot_set_deferred_append(h, on) -> None:
+    _check(lib().ipot_set_deferred_append(h, 1 if on else 0), "ipot_set_deferred_append")
 
 
 def ipot_reset(h) -> None:

@@ -64,8 +64,9 @@ def read_rotated(h, cfg: inputs.CcdConfig, rows: int) -> np.ndarray:
     return from_dev_bits(ipot.device_array(ipot.ipot_view_rope(h), shape, cfg.dtype)[:, :rows], cfg.dtype)
 
 
-def gpu_cycle(cfg: inputs.CcdConfig, t: dict, scorer=ipot.IPOT_SCORER_AUTO, n=None):
-    """Fill a fresh pot with t['K'], t['V'] (first n rows), run one cycle, read everything back."""
+def gpu_cycle(cfg: inputs.CcdConfig, t: dict, scorer=ipot.IPOT_SCORER_AUTO, n=None, deferred_from=None):
+    """Fill a fresh pot with t['K'], t['V'] (first n rows), run one cycle, read everything back.
+    deferred_from = s: rows [0, s) are appended the plain way, rows [s, n) as a deferred append."""
     n = cfg.pot_size if n is None else n
     h = make_pot(cfg, max_cap_rows=t["Q"].shape[3])
     keep_alive = []
@@ -78,7 +79,15 @@ def gpu_cycle(cfg: inputs.CcdConfig, t: dict, scorer=ipot.IPOT_SCORER_AUTO, n=No
         Kd, Vd = to_dev(t["K"][:, :, :, :n], cfg.dtype), to_dev(t["V"][:, :, :, :n], cfg.dtype)
         Qd = to_dev(t["Q"], cfg.dtype)
         auxd = torch.from_numpy(np.ascontiguousarray(t["aux"][:, :n])).cuda()
-        ipot.ipot_append_chunk(h, Kd, Vd, n)
+        if deferred_from is None:
+            ipot.ipot_append_chunk(h, Kd, Vd, n)
+        else:
+            s0 = deferred_from
+            if s0 > 0:
+                ipot.ipot_append_chunk(h, Kd[:, :, :, :s0].contiguous(), Vd[:, :, :, :s0].contiguous(), s0)
+            Kd, Vd = Kd[:, :, :, s0:].contiguous(), Vd[:, :, :, s0:].contiguous()   # alive until the cycle has run
+            ipot.ipot_set_deferred_append(h, True)
+            ipot.ipot_append_chunk(h, Kd, Vd, n - s0)
         if t.get("K_cap") is not None:  # Appendix B listing: the CaP's own keys join the softmax
             ipot.ipot_score_and_compress_cap(h, Qd, to_dev(t["K_cap"], cfg.dtype), t["Q"].shape[3],
                                              auxd if cfg.nuc_slots > 0 else None)
