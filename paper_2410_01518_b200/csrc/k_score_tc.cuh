@@ -549,11 +549,14 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                 float2 sv[16];
                 uint32_t tries = 0;
                 bool fresh;
-                do {
+#pragma unroll
+                for (int s = 0; s < 16; ++s)  // beyond the item: neutral and fresh; this CTA's own slab: known; others: stale
+                    sv[s] = (s0 + s >= tasks_per_item) ? make_float2(-INFINITY, sgn) : (s0 + s == slab) ? make_float2(ms, ls * sgn) : make_float2(0.f, 0.f);
+                do {  // only the entries that are still stale are read again
                     fresh = true;
 #pragma unroll
                     for (int s = 0; s < 16; ++s) {
-                        sv[s] = (s0 + s < tasks_per_item) ? ld_gpu_f32x2(&st[(size_t)(s0 + s) * kTcRows]) : make_float2(-INFINITY, sgn);
+                        if (!(sv[s].y * sgn > 0.f)) sv[s] = ld_gpu_f32x2(&st[(size_t)(s0 + s) * kTcRows]);
                         fresh = fresh && (sv[s].y * sgn > 0.f);
                     }
                     if (!fresh && ((++tries > kTcSpinLimit) || *ab)) {
