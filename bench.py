@@ -642,9 +642,9 @@ def main():
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["peak_source"] = pk["source"]
     roof["frac_of_nominal_8tbs"] = roof["achieved"] / 8000.0   # the HBM3e data-sheet figure, for context
-    # DRAM bytes of one launch of the scoring kernel from the committed ncu capture (profiles/): 70.745 MB for
+    # DRAM bytes of one launch of the scoring kernel from the committed ncu capture (profiles/): 71.198 MB for
     # 64 units of this shape, growing with the units; unknown for other shapes, kernels or scorers
-    roof["traffic"] = (units * 70.745e6 / 64 if dom == 1 and scorer_used == 2 and (N, M, d) == (4096, 128, 128) and not args.cap_keys else None)
+    roof["traffic"] = (units * 71.198e6 / 64 if dom == 1 and scorer_used == 2 and (N, M, d) == (4096, 128, 128) and not args.cap_keys else None)
     roof["kernel_ms"] = dict(zip(names, [round(x, 5) for x in kms]))
     roof["cycles_averaged"] = kcycles
     roof["cap_score_gbs"] = score_bytes / (kms[1] * 1e-3) / 1e9

@@ -526,16 +526,21 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
             if (prm.cap_stats && row_valid) own = __ldg(&prm.cap_stats[(size_t)(item / prm.mtiles) * prm.M + mt * kTcRows + row]);
             mbar_wait(bar(kBarEReady + b), ph, ab, prm.status);
             // ---- merge the eight chunks of the row, publish the slab's statistics
-            float cm[8];
-            float ms = -INFINITY;
+            // (this warp shares its scheduler with four busy epilogue warps and every task waits for this code: the
+            // loads are issued together and maxima and sums are folded as trees, not as chains)
+            float cm[8], ce[8];
+            {
+                float2 t[8];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                cm[i] = tstat[(b * 8 + i) * kTcRows + row].x;
-                ms = fmaxf(ms, cm[i]);  // chunk 0 always holds a valid key
+                for (int i = 0; i < 8; ++i) t[i] = tstat[(b * 8 + i) * kTcRows + row];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) cm[i] = t[i].x;
+                const float ms0 = max3(max3(cm[0], cm[1], cm[2]), max3(cm[3], cm[4], cm[5]), fmaxf(cm[6], cm[7]));  // chunk 0 always holds a valid key
+#pragma unroll
+                for (int i = 0; i < 8; ++i) ce[i] = (cm[i] == -INFINITY) ? 0.f : t[i].y * ex2(cm[i] - ms0);
             }
-            float ls = 0.f;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) ls += (cm[i] == -INFINITY) ? 0.f : tstat[(b * 8 + i) * kTcRows + row].y * ex2(cm[i] - ms);
+            const float ms = max3(max3(cm[0], cm[1], cm[2]), max3(cm[3], cm[4], cm[5]), fmaxf(cm[6], cm[7]));
+            const float ls = ((ce[0] + ce[1]) + (ce[2] + ce[3])) + ((ce[4] + ce[5]) + (ce[6] + ce[7]));
             if (tasks_per_item > 1) st_gpu_f32x2(&prm.stats[((size_t)item * tasks_per_item + slab) * kTcRows + row], ms, ls * sgn);
 
             // ---- this row's statistics of every slab of the item; re-read until all carry this launch's mark
@@ -567,12 +572,17 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                         break;
                     }
                 } while (!fresh);
-                float mb = m;
+                const float mb = max3(max3(max3(sv[0].x, sv[1].x, sv[2].x), max3(sv[3].x, sv[4].x, sv[5].x), max3(sv[6].x, sv[7].x, sv[8].x)),
+                                      max3(max3(sv[9].x, sv[10].x, sv[11].x), max3(sv[12].x, sv[13].x, sv[14].x), fmaxf(sv[15].x, m)), -INFINITY);
+                float w[16];
 #pragma unroll
-                for (int s = 0; s < 16; ++s) mb = fmaxf(mb, sv[s].x);
-                l = (m == -INFINITY) ? 0.f : l * ex2(m - mb);
+                for (int s = 0; s < 16; ++s) w[s] = fabsf(sv[s].y) * ex2(sv[s].x - mb);
 #pragma unroll
-                for (int s = 0; s < 16; ++s) l = fmaf(fabsf(sv[s].y), ex2(sv[s].x - mb), l);
+                for (int step = 1; step < 16; step <<= 1) {
+#pragma unroll
+                    for (int s = 0; s < 16; s += 2 * step) w[s] += w[s + step];
+                }
+                l = ((m == -INFINITY) ? 0.f : l * ex2(m - mb)) + w[0];
                 m = mb;
             }
             if (own.x > -INFINITY) {
@@ -580,7 +590,9 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                 l = fmaf(own.y, ex2(own.x - mb), l * ex2(m - mb));
                 m = mb;
             }
-            const float inv_l = row_valid ? 1.f / l : 0.f;
+            float inv_l;
+            asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv_l) : "f"(l));
+            if (!row_valid) inv_l = 0.f;
 #pragma unroll
             for (int i = 0; i < 8; ++i)
                 fbuf[(b * 8 + i) * kTcRows + row] = (cm[i] == -INFINITY) ? 0.f : ex2(cm[i] - m) * inv_l;
