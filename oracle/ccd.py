@@ -34,7 +34,7 @@ def _load():
         lib.ora_cycle_cap.argtypes = [dp, dp, dp, bp, bp, dp, ip, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
                                       C.c_int, C.c_int, C.c_int, C.c_size_t, dp, ip, bp, bp]
         lib.ora_token_novelty.argtypes = [dp, ip, C.c_long, C.c_int, dp]
-        lib.ora_rope_rows.argtypes = [C.c_void_p, C.c_void_p, ip, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_int]
+        lib.ora_rope_rows.argtypes = [C.c_void_p, C.c_void_p, ip, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_int, dp, dp]
         lib.ora_decode_attention.argtypes = [dp, dp, dp, C.c_int, C.c_int, C.c_int, dp, dp]
         lib.ora_set_threads.argtypes = [C.c_int]
         lib.ora_max_threads.restype = C.c_int
@@ -71,10 +71,12 @@ def max_threads() -> int:
     return int(_load().ora_max_threads())
 
 
-def rope_rows(rows, pos, cos_t, sin_t, interleaved: bool = False) -> np.ndarray:
+def rope_rows(rows, pos, cos_t, sin_t, interleaved: bool = False, with_exact: bool = False):
     """Sec. 3.4: rotary embedding of rows [..., n, d] (storage dtype: float32 or uint16 bf16 bits) at positions
     pos [n] with cos/sin tables [positions][d/2] of the same storage dtype; every leading index uses the same
-    positions.  Returns the rotated rows in the storage dtype."""
+    positions.  Computed in float64 and rounded once: returns the rotated rows in the storage dtype, and with
+    ``with_exact`` also the unrounded float64 values and the size of the two terms each value is the sum or
+    difference of (what bounds the cancellation error of a single-precision evaluation)."""
     rows = np.ascontiguousarray(rows)
     cos_t, sin_t = np.ascontiguousarray(cos_t), np.ascontiguousarray(sin_t)
     assert rows.dtype in (np.float32, np.uint16) and cos_t.dtype == rows.dtype and sin_t.dtype == rows.dtype
@@ -83,11 +85,15 @@ def rope_rows(rows, pos, cos_t, sin_t, interleaved: bool = False) -> np.ndarray:
     assert pos.shape == (n,) and d % 2 == 0 and cos_t.shape == sin_t.shape and cos_t.shape[1] == d // 2
     assert pos.min(initial=0) >= 0 and pos.max(initial=0) < cos_t.shape[0]
     out = np.empty_like(rows)
+    exact = np.empty(rows.shape, dtype=np.float64) if with_exact else None
+    mag = np.empty(rows.shape, dtype=np.float64) if with_exact else None
     flat_in, flat_out = rows.reshape(-1, n, d), out.reshape(-1, n, d)
     for i in range(flat_in.shape[0]):
+        ex = _p(exact.reshape(-1, n, d)[i], C.c_double) if with_exact else None
+        mg = _p(mag.reshape(-1, n, d)[i], C.c_double) if with_exact else None
         _load().ora_rope_rows(flat_in[i].ctypes.data, flat_out[i].ctypes.data, _p(pos, C.c_int), n, d,
-                              int(rows.dtype == np.float32), cos_t.ctypes.data, sin_t.ctypes.data, int(interleaved))
-    return out
+                              int(rows.dtype == np.float32), cos_t.ctypes.data, sin_t.ctypes.data, int(interleaved), ex, mg)
+    return (out, exact, mag) if with_exact else out
 
 
 def decode_attention(q, K, V, n: int | None = None):

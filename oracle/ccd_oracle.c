@@ -41,11 +41,10 @@
  *   - survivors keep their original order (ascending slot index);
  *   - CR-RoPE: the paper gives no rotary details.  The caller supplies cos/sin per (position,
  *     frequency) in the storage type; channel pairs are (c, c + d/2) ("half") or (2c, 2c + 1)
- *     ("interleaved"); the rotation is evaluated in single precision exactly as
- *     lo' = fma(lo, cos, -(hi * sin)), hi' = fma(hi, cos, lo * sin) and rounded once to the
- *     storage type (nearest even).  Rounding to bf16 is a quantisation, so both the checker
- *     and the CUDA path take it from the same single-precision expression; everything after
- *     it (the scores) is double precision here.
+ *     ("interleaved"); the pair is multiplied as a complex number by cos + i sin in double
+ *     precision and rounded once to the storage type (nearest even).  A CUDA path that evaluates
+ *     the same product in single precision agrees with it bit for bit except where the exact
+ *     value lies within its rounding error of a rounding boundary; the tests bound that.
  *
  *   - CaP-inclusive variant: CaP row i (0-based, within its query head) sees the
  *     CaP keys 0..i of its KV head (causal mask), all of them after every pot key;
@@ -58,9 +57,10 @@
  * columns, far-away CaP keys reduce it to ora_cap_scores, a later CaP key never
  * changes an earlier row.  Token novelty: uniform logits give log V, V = 2 is a
  * softplus, a constant added to a row changes nothing, library cross-entropy.
- * Rotary rows: position 0 is the identity, exact small cases, complex multiplication in
- * double precision, pair norms, the score of a rotated query and key depends on the
- * position difference only, the two pairings are one channel permutation apart.
+ * Rotary rows: position 0 is the identity, exact small cases, exact rational arithmetic with
+ * a brute-force search for the nearest storage value, library complex multiplication, pair
+ * norms, the score of a rotated query and key depends on the position difference only, the
+ * two pairings are one channel permutation apart.
  * Decode attention: one key returns its value, equal keys the mean value, library attention
  * and log-sum-exp, slot permutation invariance.
  */
@@ -180,54 +180,68 @@ void ora_cap_scores_incl(const double *Q, const double *K, const double *Kc, int
     free(s);
 }
 
-/* ---- storage <-> float (bf16 = upper half of a float, rounded to nearest even) ---- */
-static float ora_bf16_to_float(uint16_t b)
+/* ---- storage <-> double.  bf16 = the upper half of a float; every bf16 and float value is a double ---- */
+static double ora_load(const void *p, size_t i, int is_f32)
 {
-    uint32_t w = (uint32_t)b << 16;
+    if (is_f32) return (double)((const float *)p)[i];
+    uint32_t w = (uint32_t)((const uint16_t *)p)[i] << 16;
     float f;
     memcpy(&f, &w, 4);
-    return f;
+    return (double)f;
 }
 
-static uint16_t ora_float_to_bf16(float f)
+/* One rounding, to nearest (ties to even), from double to bf16: 8 significant bits, or a multiple of
+ * 2^-133 below the normal range. */
+static uint16_t ora_double_to_bf16(double v)
 {
+    float f;
+    if (v == 0.0 || !isfinite(v)) {
+        f = (float)v;
+    } else {
+        int e;
+        (void)frexp(fabs(v), &e);                 /* |v| = m 2^e with m in [0.5, 1) */
+        int qe = e - 8;
+        if (qe < -133) qe = -133;
+        const double q = ldexp(1.0, qe);
+        f = (float)copysign(rint(fabs(v) / q) * q, v);   /* rint: nearest even; the result fits a float exactly */
+    }
     uint32_t w;
     memcpy(&w, &f, 4);
-    w += 0x7FFFu + ((w >> 16) & 1u);
     return (uint16_t)(w >> 16);
 }
 
-static float ora_load(const void *p, size_t i, int is_f32)
+static void ora_store(void *p, size_t i, int is_f32, double v)
 {
-    return is_f32 ? ((const float *)p)[i] : ora_bf16_to_float(((const uint16_t *)p)[i]);
-}
-
-static void ora_store(void *p, size_t i, int is_f32, float v)
-{
-    if (is_f32) ((float *)p)[i] = v;
-    else ((uint16_t *)p)[i] = ora_float_to_bf16(v);
+    if (is_f32) ((float *)p)[i] = (float)v;       /* one rounding to nearest even */
+    else ((uint16_t *)p)[i] = ora_double_to_bf16(v);
 }
 
 /*
  * Sec. 3.4: rotary embedding of n rows of d channels; row r gets position pos[r].  cos_t and
  * sin_t are [positions][d/2] tables in the storage type.  interleaved = 0 pairs channel c with
- * c + d/2, 1 pairs 2c with 2c + 1; frequency index c in both.  in and out may not overlap.
+ * c + d/2, 1 pairs 2c with 2c + 1; frequency index c in both.  Each pair (lo, hi) is the complex
+ * number lo + i hi multiplied by cos + i sin, in double precision (the products of two storage
+ * values are exact there), rounded once to the storage type.  in and out may not overlap.
+ * exact and mag (each may be NULL, [n][d] doubles) receive the unrounded result and
+ * |lo cos| + |hi sin| resp. |hi cos| + |lo sin|: the size of the terms whose difference the
+ * result is, which bounds what an evaluation in a narrower type can lose to cancellation.
  */
 void ora_rope_rows(const void *in, void *out, const int *pos, int n, int d, int is_f32,
-                   const void *cos_t, const void *sin_t, int interleaved)
+                   const void *cos_t, const void *sin_t, int interleaved, double *exact, double *mag)
 {
     const int half = d / 2;
     for (int r = 0; r < n; ++r) {
         for (int c = 0; c < half; ++c) {
             const size_t ilo = (size_t)r * d + (interleaved ? 2 * c : c);
             const size_t ihi = (size_t)r * d + (interleaved ? 2 * c + 1 : c + half);
-            const float lo = ora_load(in, ilo, is_f32), hi = ora_load(in, ihi, is_f32);
-            const float cs = ora_load(cos_t, (size_t)pos[r] * half + c, is_f32);
-            const float sn = ora_load(sin_t, (size_t)pos[r] * half + c, is_f32);
-            volatile float t1 = hi * sn;   /* volatile: each product is rounded on its own */
-            volatile float t2 = lo * sn;
-            ora_store(out, ilo, is_f32, fmaf(lo, cs, -t1));
-            ora_store(out, ihi, is_f32, fmaf(hi, cs, t2));
+            const double lo = ora_load(in, ilo, is_f32), hi = ora_load(in, ihi, is_f32);
+            const double cs = ora_load(cos_t, (size_t)pos[r] * half + c, is_f32);
+            const double sn = ora_load(sin_t, (size_t)pos[r] * half + c, is_f32);
+            const double re = lo * cs - hi * sn, im = hi * cs + lo * sn;
+            ora_store(out, ilo, is_f32, re);
+            ora_store(out, ihi, is_f32, im);
+            if (exact) { exact[ilo] = re; exact[ihi] = im; }
+            if (mag) { mag[ilo] = fabs(lo * cs) + fabs(hi * sn); mag[ihi] = fabs(hi * cs) + fabs(lo * sn); }
         }
     }
 }

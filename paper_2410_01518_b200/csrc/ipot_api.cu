@@ -753,7 +753,7 @@ int ipot_nuc_scores(ipot_t *p, const void *logits, int logits_dtype, long long r
     const size_t need = rows * ((vocab + kNovSegElems - 1) / kNovSegElems);
     if (!p->nov_scratch || need > p->nov_capacity) {  // first use or a larger shape: the only allocation outside ipot_create
         IPOT_CUDA(cudaStreamSynchronize(p->stream));
-        cudaFree(p->nov_scratch); cudaFree(p->dec_partial); cudaFree(p->dec_counters);
+        cudaFree(p->nov_scratch);  // only this call's own scratch: every other buffer keeps its owner
         p->nov_scratch = nullptr;
         p->nov_capacity = 0;
         if (cudaMalloc((void **)&p->nov_scratch, kNovCounterBytes + need * sizeof(float2)) != cudaSuccess) {

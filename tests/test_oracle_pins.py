@@ -387,13 +387,62 @@ def test_rope_is_complex_multiplication():
     cos_t, sin_t = _tables(64, d)
     rows = g.standard_normal((n, d)).astype(np.float32)
     pos = g.integers(0, 64, n)
-    out = oracle.rope_rows(rows, pos, cos_t, sin_t).astype(np.float64)
+    out, exact, mag = oracle.rope_rows(rows, pos, cos_t, sin_t, with_exact=True)
     z = rows[:, :d // 2].astype(np.float64) + 1j * rows[:, d // 2:].astype(np.float64)
-    w = z * (cos_t[pos].astype(np.float64) + 1j * sin_t[pos].astype(np.float64))
-    np.testing.assert_allclose(out[:, :d // 2], w.real, rtol=0, atol=2e-6)
-    np.testing.assert_allclose(out[:, d // 2:], w.imag, rtol=0, atol=2e-6)
+    w = z * (cos_t[pos].astype(np.float64) + 1j * sin_t[pos].astype(np.float64))        # the library's complex product
+    assert (exact[:, :d // 2] == w.real).all() and (exact[:, d // 2:] == w.imag).all()
+    assert (out[:, :d // 2] == w.real.astype(np.float32)).all() and (out[:, d // 2:] == w.imag.astype(np.float32)).all()
+    a, b = np.abs(rows[:, :d // 2].astype(np.float64)), np.abs(rows[:, d // 2:].astype(np.float64))
+    c, s_ = np.abs(cos_t[pos].astype(np.float64)), np.abs(sin_t[pos].astype(np.float64))
+    assert (mag[:, :d // 2] == a * c + b * s_).all() and (mag[:, d // 2:] == b * c + a * s_).all()
     # pair norms survive the rotation (up to the table's rounding)
-    np.testing.assert_allclose(out[:, :d // 2] ** 2 + out[:, d // 2:] ** 2, np.abs(z) ** 2, rtol=1e-5)
+    o = out.astype(np.float64)
+    np.testing.assert_allclose(o[:, :d // 2] ** 2 + o[:, d // 2:] ** 2, np.abs(z) ** 2, rtol=1e-5)
+
+
+def test_rope_rounds_the_exact_product_once_to_the_nearest_storage_value():
+    """Exact rational arithmetic, then a brute-force search over every finite bf16 value for the nearest one
+    (ties: even bit pattern).  A product rounded through float32 first would fail the constructed tie case."""
+    from fractions import Fraction
+    from paper_2410_01518_b200 import inputs
+    g = rnd(75)
+    d, n = 12, 9
+    rows = g.standard_normal((n, d)).astype(np.float32)
+    pos = g.integers(0, 32, n)
+    rb, cb, sb = inputs.store(rows, "bf16"), *inputs.make_rope_table(32, d, "bf16")
+    got = oracle.rope_rows(rb, pos, cb, sb)
+    bits = np.arange(65536, dtype=np.uint32)
+    with np.errstate(invalid="ignore"):
+        vals = (bits << np.uint32(16)).view(np.float32).astype(np.float64)
+    finite = np.isfinite(vals)
+
+    def nearest(x: Fraction) -> int:
+        xf = float(x)                                   # exact: a sum of two 16-bit products
+        assert Fraction(xf) == x
+        dist = np.where(finite, np.abs(vals - xf), np.inf)
+        best = np.flatnonzero(dist == dist.min())
+        if xf == 0.0:
+            return 0
+        best = [b for b in best if (vals[b] >= 0) == (xf >= 0) or vals[b] == 0]
+        return int(min(best, key=lambda b: b & 1))      # a tie has one even and one odd neighbour
+
+    w = lambda a: Fraction(float(inputs.widen(np.array([a], dtype=np.uint16), "bf16")[0]))
+    for r in range(n):
+        for c in range(d // 2):
+            lo, hi, cs, sn = w(rb[r, c]), w(rb[r, c + d // 2]), w(cb[pos[r], c]), w(sb[pos[r], c])
+            assert int(got[r, c]) == nearest(lo * cs - hi * sn)
+            assert int(got[r, c + d // 2]) == nearest(hi * cs + lo * sn)
+    # a case that rounding through float32 first gets wrong: lo cos - hi sin = (1 + 2^-7)(1 - 2^-8) + 145 * 113 * 2^-29
+    # = 1 + 2^-8 + 2^-29, just above the midpoint of the bf16 neighbours 1 and 1 + 2^-7.  float32 drops the 2^-29,
+    # lands on the midpoint and would then tie to even (1.0); one rounding from the exact value gives 1 + 2^-7.
+    x = inputs.store(np.array([[1.0 + 2.0 ** -7, -145.0 * 2.0 ** -14]], dtype=np.float32), "bf16")
+    ct = inputs.store(np.array([[1.0 - 2.0 ** -8]], dtype=np.float32), "bf16")
+    st = inputs.store(np.array([[113.0 * 2.0 ** -15]], dtype=np.float32), "bf16")
+    val = Fraction(1) + Fraction(1, 2 ** 8) + Fraction(1, 2 ** 29)
+    assert w(x[0, 0]) * w(ct[0, 0]) - w(x[0, 1]) * w(st[0, 0]) == val
+    assert nearest(val) == 0x3F81
+    assert int(oracle.rope_rows(x, [0], ct, st)[0, 0]) == 0x3F81
+    assert int(inputs.store(np.array([np.float32(float(val))]), "bf16")[0]) == 0x3F80   # the two-step route differs
 
 
 def test_rope_scores_depend_on_the_position_difference():
@@ -410,7 +459,7 @@ def test_rope_scores_depend_on_the_position_difference():
     assert abs(other - dots[0]) > 1e-3                                                  # and on nothing less
 
 
-def test_rope_pairings_are_a_channel_permutation_apart_and_bf16_rounds_once():
+def test_rope_pairings_are_a_channel_permutation_apart():
     g = rnd(73)
     d, n = 12, 9
     rows = g.standard_normal((n, d)).astype(np.float32)
@@ -422,13 +471,6 @@ def test_rope_pairings_are_a_channel_permutation_apart_and_bf16_rounds_once():
     inter = oracle.rope_rows(inter_in, pos, cos_t, sin_t, True)
     ref = oracle.rope_rows(rows, pos, cos_t, sin_t, False)
     assert (inter[:, 0::2] == ref[:, :d // 2]).all() and (inter[:, 1::2] == ref[:, d // 2:]).all()
-    # bf16 storage: the float32 result rounded once to nearest even
-    from paper_2410_01518_b200 import inputs
-    rb, cb, sb = inputs.store(rows, "bf16"), *inputs.make_rope_table(32, d, "bf16")
-    got = oracle.rope_rows(rb, pos, cb, sb)
-    f = oracle.rope_rows(inputs.widen(rb, "bf16").astype(np.float32), pos, inputs.widen(cb, "bf16").astype(np.float32),
-                         inputs.widen(sb, "bf16").astype(np.float32))
-    assert (got == inputs.store(f, "bf16")).all()
 
 
 def test_cycle_with_rope_scores_rotated_keys_and_moves_unrotated_rows():

@@ -1,14 +1,15 @@
 """GPU parity of the context-reset rotary mode (Sec. 3.4): unrotated keys in the pot, a rotated copy kept by the
-row movers, scores from the rotated copy - against the CPU checker, through the C ABI.  The rotated rows are
-compared bit for bit (both sides round the same single-precision expression once); scores and index lists under
-the tolerances of tests/parity.py."""
+row movers, scores from the rotated copy - against the CPU checker, through the C ABI.  The checker rotates in
+float64 and rounds once; the rotated rows must lie within the error bound of the kernel's single-precision
+evaluation and be bit-equal almost everywhere (tests/parity.py states both numbers); scores and index lists
+under the tolerances of tests/parity.py."""
 import numpy as np
 import pytest
 import torch
 
 import oracle
 from paper_2410_01518_b200 import inputs, ipot
-from parity import compare_cycle, from_dev_bits, gpu_cycle, make_pot, read_results, read_rotated, to_dev
+from parity import check_rotated, compare_cycle, from_dev_bits, gpu_cycle, make_pot, read_results, read_rotated, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -92,7 +93,7 @@ def test_stream_of_cycles_keeps_the_rotated_copy_current():
             pot_v = from_dev_bits(ipot.device_array(Vp, shape, "bf16"), "bf16")
             assert (pot_k[:, filled:] == Kn.reshape(cfg.units, n_new, cfg.d)).all()
             rot = read_rotated(h, cfg, cfg.pot_size)
-            assert (rot == oracle.rope_rows(pot_k, np.arange(cfg.pot_size), cos_t, sin_t)).all()
+            check_rotated(rot, pot_k, np.arange(cfg.pot_size), (cos_t, sin_t, False), "bf16")
             t = {"K": pot_k.reshape(cfg.layers, cfg.batch, cfg.Hkv, cfg.pot_size, cfg.d),
                  "V": pot_v.reshape(cfg.layers, cfg.batch, cfg.Hkv, cfg.pot_size, cfg.d),
                  "Q": inputs.make_q(cfg, step), "aux": inputs.make_aux(cfg, step), "rope": (cos_t, sin_t, False)}
@@ -132,6 +133,6 @@ def test_enable_rope_argument_and_state_errors():
         ipot.ipot_enable_rope(h, c, s, ipot.IPOT_ROPE_INTERLEAVED)
         ipot.ipot_append_chunk(h, to_dev(K, "bf16"), to_dev(V, "bf16"), 32)
         rot = read_rotated(h, cfg, 32)
-        assert (rot == oracle.rope_rows(K.reshape(cfg.units, 32, 64), np.arange(32), cos_t, sin_t, True)).all()
+        check_rotated(rot, K.reshape(cfg.units, 32, 64), np.arange(32), (cos_t, sin_t, True), "bf16")
     finally:
         ipot.ipot_destroy(h)
