@@ -116,33 +116,36 @@ def test_tensor_scorer_shapes(case):
     np.testing.assert_allclose(gpu[0], simt[0], rtol=2e-5, atol=1e-30)  # the two GPU scorers agree far inside 1e-3
 
 
-def test_config3_full_size_sampled_units():
-    """All 32 layers in one call (the launch the benchmark times); the checker follows 12 sampled units."""
+def test_config3_full_size_every_unit():
+    """All 32 layers in one call (the launch the benchmark times); the checker follows every one of the 256 units."""
     cfg = inputs.CONFIGS[3]
     K0, V0 = inputs.make_kv(cfg, 2048, chunk=0)
     K1, V1 = inputs.make_kv(cfg, 2048, chunk=1)
     t = {"K": np.concatenate([K0, K1], axis=3), "V": np.concatenate([V0, V1], axis=3),
          "Q": inputs.make_q(cfg, 1), "aux": inputs.make_aux(cfg, 1)}
     gpu = gpu_cycle(cfg, t, ipot.IPOT_SCORER_AUTO)
-    units = np.linspace(0, cfg.units - 1, 12).astype(np.int32)
-    same, cnt = compare_cycle(cfg, t, gpu, units=units)
-    assert cnt == 12 and same >= 11
+    same, cnt = compare_cycle(cfg, t, gpu)
+    # adjacent order statistics of 4096 scores lie ~3e-4 apart relatively and the decision is taken in fp32 on the
+    # GPU, so a unit in a few hundred may resolve its last slot the other way (inside the tie band, checked per slot)
+    assert cnt == cfg.units and same >= cnt - 3
     u, idx = gpu[0], gpu[1]
     assert np.abs(u.sum(axis=1) - cfg.G * cfg.cap_rows).max() < 2e-2      # holds at any size
     assert (np.diff(idx, axis=1) > 0).all() and idx.min() >= 0 and idx.max() < cfg.pot_size
 
 
-@pytest.mark.parametrize("cfg_id,n_sample", [(4, 8), (5, 6)])
+@pytest.mark.parametrize("cfg_id,n_sample", [(4, 32), (5, 32)])
 def test_configs_4_and_5_full_size_sampled_units(cfg_id, n_sample):
     """Llama-3-8B-shaped batch of 16 streams (pot 8192, 2 row blocks) and the 70B-shaped layer (pot 16384,
     4 row blocks, heavy-tailed keys, 5 % exactly duplicated tokens): the whole configuration runs on the
-    GPU, the checker follows sampled units; properties that hold at any size are checked on all units."""
+    GPU, the checker follows 32 units spread over all streams and heads; properties that hold at any size are
+    checked on all units.  Every unit whose list differs from the checker's differs only in slots inside the
+    tie band (asserted per slot by compare_cycle); at most one followed unit in eight may do so."""
     cfg = inputs.CONFIGS[cfg_id]
     t = inputs.make_cycle(cfg)
     gpu = gpu_cycle(cfg, t, ipot.IPOT_SCORER_AUTO)
-    units = np.linspace(0, cfg.units - 1, n_sample).astype(np.int32)
+    units = np.unique(np.concatenate([np.linspace(0, cfg.units - 1, n_sample - 2).astype(np.int32), [1, cfg.units - 2]]))
     same, cnt = compare_cycle(cfg, t, gpu, units=units)
-    assert cnt == n_sample and same >= n_sample - 2
+    assert cnt >= n_sample - 2 and same >= cnt - cnt // 8
     u, idx, K, V = gpu
     M = cfg.G * cfg.cap_rows
     assert np.abs(u.sum(axis=1) - M).max() < 1e-4 * M
@@ -154,6 +157,54 @@ def test_configs_4_and_5_full_size_sampled_units(cfg_id, n_sample):
         nuc = set(oracle.nuc_top(t["aux"][b], cfg.nuc_slots).tolist())
         for g in range(cfg.Hkv):
             assert nuc <= set(idx[b * cfg.Hkv + g].tolist())
+
+
+@pytest.mark.parametrize("deferred", [False, True])
+def test_config3_full_size_stream_of_cycles(deferred):
+    """The 32-layer stream at full size through three consecutive fill/distil rounds (Sec. 3.2), with the plain and
+    with the deferred append.  The checker keeps its own pot for 40 units (the first and last eight and 24 spread
+    over the layers); after every cycle scores, index lists and the pot's K, V bytes are compared, and the checker's
+    pot is advanced with the validated GPU lists.  What a launch carries over to the next one (survivor rows, the
+    deferred chunk, scorer state) is thereby followed at the shape the benchmark times."""
+    cfg = inputs.CONFIGS[3]
+    N, keep, d = cfg.pot_size, cfg.keep, cfg.d
+    units = np.unique(np.concatenate([np.arange(8), np.arange(cfg.units - 8, cfg.units),
+                                      np.linspace(8, cfg.units - 9, 24).astype(np.int64)])).astype(np.int32)
+    shape5 = (cfg.layers, cfg.batch, cfg.Hkv)
+    h = make_pot(cfg)
+    alive = []
+    try:
+        if deferred:
+            ipot.ipot_set_deferred_append(h, True)
+        K0, V0 = inputs.make_kv(cfg, N - keep, chunk=0)
+        alive.append((to_dev(K0, "bf16"), to_dev(V0, "bf16")))
+        ipot.ipot_append_chunk(h, alive[-1][0], alive[-1][1], N - keep)
+        refK = K0.reshape(cfg.units, N - keep, d)[units]       # the checker's pot, followed units only
+        refV = V0.reshape(cfg.units, N - keep, d)[units]
+        for cyc in range(1, 4):
+            Kc, Vc = inputs.make_kv(cfg, N - refK.shape[1], chunk=cyc)
+            alive.append((to_dev(Kc, "bf16"), to_dev(Vc, "bf16")))      # a deferred chunk is read where it lies
+            ipot.ipot_append_chunk(h, alive[-1][0], alive[-1][1], Kc.shape[3])
+            fullK = np.zeros((cfg.units, N, d), dtype=np.uint16)
+            fullV = np.zeros((cfg.units, N, d), dtype=np.uint16)
+            fullK[units] = np.concatenate([refK, Kc.reshape(cfg.units, -1, d)[units]], axis=1)
+            fullV[units] = np.concatenate([refV, Vc.reshape(cfg.units, -1, d)[units]], axis=1)
+            t = {"K": fullK.reshape(shape5 + (N, d)), "V": fullV.reshape(shape5 + (N, d)),
+                 "Q": inputs.make_q(cfg, cyc), "aux": inputs.make_aux(cfg, cyc)}
+            ipot.ipot_score_and_compress(h, to_dev(t["Q"], "bf16"), cfg.cap_rows, torch.from_numpy(t["aux"]).cuda())
+            u, idx, K, V = read_results(h, cfg, N)
+            same, cnt = compare_cycle(cfg, t, (u, idx, K, V), units=units)
+            assert cnt == len(units) and same >= cnt - 2, (cyc, same)
+            assert np.abs(u.sum(axis=1) - cfg.G * cfg.cap_rows).max() < 2e-2
+            assert (np.diff(idx, axis=1) > 0).all() and idx.min() >= 0 and idx.max() < N
+            refK = np.stack([oracle.gather(fullK[unit], idx[unit]) for unit in units])
+            refV = np.stack([oracle.gather(fullV[unit], idx[unit]) for unit in units])
+            assert (K[units] == refK).all() and (V[units] == refV).all()
+            Kp, Vp, ln = ipot.ipot_view(h)
+            assert ln == keep
+            del alive[:-1]                                               # older chunks are in the pot by now
+    finally:
+        ipot.ipot_destroy(h)
 
 
 def test_partially_filled_pot():
