@@ -68,8 +68,12 @@ enum {
     IPOT_SCORER_AUTO = 0,   /* the fastest kernel the shape allows: tcgen05, else warp-level tensor cores, else fp32 FMAs */
     IPOT_SCORER_SIMT = 1,   /* fp32 FMA kernel: any supported shape, f32 or bf16 */
     IPOT_SCORER_TENSOR = 2, /* tcgen05 kernel (bf16, d = 64 or 128): IPOT_E_INVALID if the shape does not allow it */
-    IPOT_SCORER_WARP_MMA = 3 /* warp-level tensor-core kernels (bf16, d a multiple of 16): what AUTO takes for bf16
+    IPOT_SCORER_WARP_MMA = 3, /* warp-level tensor-core kernels (bf16, d a multiple of 16): what AUTO takes for bf16
                                 pots the tcgen05 kernel does not; IPOT_E_INVALID if the shape does not allow it */
+    IPOT_SCORER_TENSOR_SWEEPS = 4 /* tcgen05 kernel that goes over the keys twice (row log-sum-exps, then probabilities
+                                and their column sums) inside thread-block clusters, so that no block waits for a block
+                                it is not co-scheduled with (bf16, d = 64 or 128, at most 512 folded query rows):
+                                IPOT_E_INVALID if the shape does not allow it */
 };
 
 typedef struct {
@@ -103,8 +107,29 @@ int ipot_set_stream(ipot_t *pot, void *cuda_stream);
 /* Sec. 3.3.3 / Sec. 4.4.2: number of slots T given to the novelty ranking, 0 <= T <= keep. */
 int ipot_set_nuc_slots(ipot_t *pot, int T);
 
-/* IPOT_SCORER_*; TENSOR is refused at the next cycle if the shape does not allow it. */
+/* IPOT_SCORER_*; a tensor-core scorer is refused at the next cycle if the shape does not allow it. */
 int ipot_set_scorer(ipot_t *pot, int scorer);
+
+/*
+ * Launch parameters of the scoring kernels (Eq. 2 itself is not affected; results stay within the stated
+ * tolerances for every setting).  `what`:
+ *   IPOT_TUNE_SWEEPS_CLUSTER      CTAs per thread-block cluster of IPOT_SCORER_TENSOR_SWEEPS: 1, 2, 4, 8, or 0 = chosen
+ *                                 from the shape (the default)
+ *   IPOT_TUNE_SWEEPS_FMA_EIGHTHS  how many eighths of that kernel's exponentials are evaluated as a polynomial on the
+ *                                 FMA pipe instead of the special-function unit: 0, 2, 3, 4, or -1 = default
+ *   IPOT_TUNE_WAIT_LIMIT_NS       time after which a device-side wait of that kernel gives up and the launch ends with
+ *                                 IPOT_E_TIMEOUT in the status word (default 200 ms; at least 1000)
+ *   IPOT_TUNE_TEST_WITHHOLD_RANK  for tests of the give-up path only: CTA `value` (0-7) of every cluster never reports
+ *                                 its row statistics, so every wait for them runs into the limit; -1 = off (default)
+ * Errors: INVALID (unknown `what`, value out of range).  Takes effect at the next launch.
+ */
+enum {
+    IPOT_TUNE_SWEEPS_CLUSTER = 1,
+    IPOT_TUNE_SWEEPS_FMA_EIGHTHS = 2,
+    IPOT_TUNE_WAIT_LIMIT_NS = 3,
+    IPOT_TUNE_TEST_WITHHOLD_RANK = 4
+};
+int ipot_set_tuning(ipot_t *pot, int what, long long value);
 
 /* Forget the contents: len = 0.  Nothing is launched.  Also the way back to a defined state after
  * ipot_sync_status() reported IPOT_E_TIMEOUT: the scorer's exchange buffers are cleared before their next use

@@ -18,6 +18,7 @@
 #include "k_score_mma.cuh"
 #include "k_score_simt.cuh"
 #include "k_score_tc.cuh"
+#include "k_score_ts.cuh"
 #include "k_select.cuh"
 
 using namespace ipotk;
@@ -73,6 +74,8 @@ struct ipot {
     int ev_used;
     long long launches;
     TcPlan tc;           // tensor-core scorer state
+    TsTuning ts;         // launch parameters of the two-sweep tensor-core scorer
+    TsOccupancy ts_occ;
 };
 
 namespace {
@@ -217,6 +220,19 @@ int launch_warp_mma(ipot *p, const void *Q, const float2 *cap_stats, int M, int 
     return IPOT_OK;
 }
 
+// The fastest scorer the shape allows.
+int auto_scorer(const ipot *p, int N, int M, bool tc_ok, bool ts_ok, bool mma_ok)
+{
+    (void)p;
+    (void)N;
+    // measured on the three-to-four-row-block shapes (M = 384, 512): the two-sweep kernel holds every query tile of a
+    // unit against a key slab that is fetched once per sweep and is 1.4 x faster there; up to two row blocks the
+    // one-sweep kernel with its statistics exchange is as fast or faster
+    if (ts_ok && (!tc_ok || M > 2 * kTcRows)) return IPOT_SCORER_TENSOR_SWEEPS;
+    if (tc_ok) return IPOT_SCORER_TENSOR;
+    return mma_ok ? IPOT_SCORER_WARP_MMA : IPOT_SCORER_SIMT;
+}
+
 // Steps 1-2 (and the timing events around them).  On success *parts tells how many
 // partial score arrays the scorer wrote.
 int run_scoring(ipot *p, const void *Q, const void *Kc, int cap_rows, const float *aux, int *parts)
@@ -224,13 +240,16 @@ int run_scoring(ipot *p, const void *Q, const void *Kc, int cap_rows, const floa
     const int N = p->len, T = p->cfg.nuc_slots, M = p->G * cap_rows;
     int scorer = p->scorer;
     const bool tc_ok = tc_applicable(p->tc, p->cfg, N, M);
+    const bool ts_ok = ts_applicable(p->tc, p->cfg, N, M);
     const bool mma_ok = p->cfg.dtype == IPOT_BF16 && p->cfg.d % 16 == 0;
     if (scorer == IPOT_SCORER_TENSOR && !tc_ok) return IPOT_E_INVALID;
+    if (scorer == IPOT_SCORER_TENSOR_SWEEPS && !ts_ok) return IPOT_E_INVALID;
     if (scorer == IPOT_SCORER_WARP_MMA && !mma_ok) return IPOT_E_INVALID;
-    if (scorer == IPOT_SCORER_AUTO) scorer = tc_ok ? IPOT_SCORER_TENSOR : mma_ok ? IPOT_SCORER_WARP_MMA : IPOT_SCORER_SIMT;
-    // keys of a deferred append: the tensor-core scorer reads whole slabs of them where they are, anything else
+    if (scorer == IPOT_SCORER_AUTO) scorer = auto_scorer(p, N, M, tc_ok, ts_ok, mma_ok);
+    // keys of a deferred append: the tensor-core scorers read whole slabs of them where they are, anything else
     // wants them in the pot
-    const bool keys_in_chunk = p->pend_K && scorer == IPOT_SCORER_TENSOR && p->pend_first % kTcSlab == 0;
+    const int slab_keys = scorer == IPOT_SCORER_TENSOR ? kTcSlab : scorer == IPOT_SCORER_TENSOR_SWEEPS ? kTsSlab : 0;
+    const bool keys_in_chunk = p->pend_K && slab_keys && p->pend_first % slab_keys == 0;
     if (p->pend_K && !keys_in_chunk) {
         int mrc = materialise(p, true, false);
         if (mrc != IPOT_OK) return mrc;
@@ -256,6 +275,10 @@ int run_scoring(ipot *p, const void *Q, const void *Kc, int cap_rows, const floa
         rc = tc_launch(p->tc, p->cfg, Q, score_keys(p), cap_stats, p->scores, (size_t)p->units * p->cfg.pot_size, N, M, p->units, p->status,
                        p->stream, parts, &n_launch, keys_in_chunk ? p->pend_K : nullptr, keys_in_chunk ? p->pend_first : 0);
         p->launches += n_launch;
+    } else if (scorer == IPOT_SCORER_TENSOR_SWEEPS) {
+        rc = ts_launch(p->tc, p->ts_occ, p->ts, p->cfg, Q, score_keys(p), cap_stats, p->scores, N, M, p->units, p->status, p->stream,
+                       keys_in_chunk ? p->pend_K : nullptr, keys_in_chunk ? p->pend_first : 0);
+        p->launches += 1;
     } else if (scorer == IPOT_SCORER_WARP_MMA) {
         rc = launch_warp_mma(p, Q, cap_stats, M, N);
     } else {
@@ -578,9 +601,34 @@ int ipot_set_nuc_slots(ipot_t *p, int T)
 
 int ipot_set_scorer(ipot_t *p, int scorer)
 {
-    if (!p || scorer < IPOT_SCORER_AUTO || scorer > IPOT_SCORER_WARP_MMA) return IPOT_E_INVALID;
+    if (!p || scorer < IPOT_SCORER_AUTO || scorer > IPOT_SCORER_TENSOR_SWEEPS) return IPOT_E_INVALID;
     p->scorer = scorer;
     return IPOT_OK;
+}
+
+int ipot_set_tuning(ipot_t *p, int what, long long value)
+{
+    if (!p) return IPOT_E_INVALID;
+    switch (what) {
+    case IPOT_TUNE_SWEEPS_CLUSTER:
+        if (value != 0 && value != 1 && value != 2 && value != 4 && value != 8) return IPOT_E_INVALID;
+        p->ts.cluster = (int)value;
+        return IPOT_OK;
+    case IPOT_TUNE_SWEEPS_FMA_EIGHTHS:
+        if (value != -1 && value != 2 && value != 3) return IPOT_E_INVALID;
+        p->ts.poly = (int)value;
+        return IPOT_OK;
+    case IPOT_TUNE_WAIT_LIMIT_NS:
+        if (value < 1000) return IPOT_E_INVALID;
+        p->ts.wait_ns = (unsigned long long)value;
+        return IPOT_OK;
+    case IPOT_TUNE_TEST_WITHHOLD_RANK:
+        if (value < -1 || value > 7) return IPOT_E_INVALID;
+        p->ts.withhold_rank = (int)value;
+        return IPOT_OK;
+    default:
+        return IPOT_E_INVALID;
+    }
 }
 
 int ipot_set_deferred_append(ipot_t *p, int on)

@@ -19,7 +19,8 @@ from . import build as _build
 IPOT_OK, IPOT_E_INVALID, IPOT_E_STATE, IPOT_E_NOMEM, IPOT_E_CUDA, IPOT_E_TIMEOUT, IPOT_E_BOUNDS, IPOT_E_LIMIT = 0, -1, -2, -3, -4, -5, -6, -7
 IPOT_NOALLOC_MAX_ROWS = 65536
 IPOT_BF16, IPOT_F32 = 0, 1
-IPOT_SCORER_AUTO, IPOT_SCORER_SIMT, IPOT_SCORER_TENSOR, IPOT_SCORER_WARP_MMA = 0, 1, 2, 3
+IPOT_SCORER_AUTO, IPOT_SCORER_SIMT, IPOT_SCORER_TENSOR, IPOT_SCORER_WARP_MMA, IPOT_SCORER_TENSOR_SWEEPS = 0, 1, 2, 3, 4
+IPOT_TUNE_SWEEPS_CLUSTER, IPOT_TUNE_SWEEPS_FMA_EIGHTHS, IPOT_TUNE_WAIT_LIMIT_NS, IPOT_TUNE_TEST_WITHHOLD_RANK = 1, 2, 3, 4
 IPOT_ROPE_HALF, IPOT_ROPE_INTERLEAVED = 1, 2
 
 # every symbol include/ipot.h declares
@@ -31,7 +32,7 @@ SYMBOLS = [
     "ipot_kernel_ms", "ipot_launch_count", "ipot_strerror", "ipot_cap_scores_noalloc",
     "ipot_score_and_compress_cap", "ipot_score_only_cap", "ipot_score_and_compress_cap_host",
     "ipot_nuc_scores", "ipot_enable_rope", "ipot_view_rope",
-    "ipot_decode_attention",
+    "ipot_decode_attention", "ipot_set_tuning",
 ]
 
 
@@ -70,6 +71,7 @@ def lib() -> C.CDLL:
         L.ipot_set_nuc_slots.argtypes = [vp, ip]
         L.ipot_set_scorer.argtypes = [vp, ip]
         L.ipot_set_deferred_append.argtypes = [vp, ip]
+        L.ipot_set_tuning.argtypes = [vp, ip, C.c_longlong]
         L.ipot_reset.argtypes = [vp]
         L.ipot_append_chunk.argtypes = [vp, vp, vp, ip]
         L.ipot_append_chunk_host.argtypes = [vp, vp, vp, ip]
@@ -148,6 +150,10 @@ def ipot_set_nuc_slots(h, T) -> None:
 
 def ipot_set_scorer(h, scorer) -> None:
     _check(lib().ipot_set_scorer(h, scorer), "ipot_set_scorer")
+
+
+def ipot_set_tuning(h, what, value) -> None:
+    _check(lib().ipot_set_tuning(h, what, value), "ipot_set_tuning")
 
 
 def ipot_set_deferred_append(h, on) -> None:

@@ -89,14 +89,17 @@ def check_rotated(got: np.ndarray, rows: np.ndarray, pos, rope, dtype: str) -> f
     return frac
 
 
-def gpu_cycle(cfg: inputs.CcdConfig, t: dict, scorer=ipot.IPOT_SCORER_AUTO, n=None, deferred_from=None):
+def gpu_cycle(cfg: inputs.CcdConfig, t: dict, scorer=ipot.IPOT_SCORER_AUTO, n=None, deferred_from=None, tuning=None):
     """Fill a fresh pot with t['K'], t['V'] (first n rows), run one cycle, read everything back.
-    deferred_from = s: rows [0, s) are appended the plain way, rows [s, n) as a deferred append."""
+    deferred_from = s: rows [0, s) are appended the plain way, rows [s, n) as a deferred append.
+    tuning: {IPOT_TUNE_*: value} launch parameters set before the cycle."""
     n = cfg.pot_size if n is None else n
     h = make_pot(cfg, max_cap_rows=t["Q"].shape[3])
     keep_alive = []
     try:
         ipot.ipot_set_scorer(h, scorer)
+        for what, value in (tuning or {}).items():
+            ipot.ipot_set_tuning(h, what, value)
         if t.get("rope") is not None:  # Sec. 3.4: t["K"] holds unrotated keys, the library keeps the rotated copy
             cos_t, sin_t, inter = t["rope"]
             keep_alive = [to_dev(cos_t, cfg.dtype), to_dev(sin_t, cfg.dtype)]
