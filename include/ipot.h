@@ -116,11 +116,14 @@ int ipot_set_scorer(ipot_t *pot, int scorer);
  *   IPOT_TUNE_SWEEPS_CLUSTER      CTAs per thread-block cluster of IPOT_SCORER_TENSOR_SWEEPS: 1, 2, 4, 8, or 0 = chosen
  *                                 from the shape (the default)
  *   IPOT_TUNE_SWEEPS_FMA_EIGHTHS  how many eighths of that kernel's exponentials are evaluated as a polynomial on the
- *                                 FMA pipe instead of the special-function unit: 0, 2, 3, 4, or -1 = default
- *   IPOT_TUNE_WAIT_LIMIT_NS       time after which a device-side wait of that kernel gives up and the launch ends with
- *                                 IPOT_E_TIMEOUT in the status word (default 200 ms; at least 1000)
- *   IPOT_TUNE_TEST_WITHHOLD_RANK  for tests of the give-up path only: CTA `value` (0-7) of every cluster never reports
- *                                 its row statistics, so every wait for them runs into the limit; -1 = off (default)
+ *                                 FMA pipe instead of the special-function unit: 2, 3, or -1 = default
+ *   IPOT_TUNE_WAIT_LIMIT_NS       time after which a device-side wait of a tensor-core scorer gives up and the launch
+ *                                 ends with IPOT_E_TIMEOUT in the status word (default 200 ms; at least 1000).
+ *                                 IPOT_SCORER_TENSOR_SWEEPS counts it from the start of each wait, IPOT_SCORER_TENSOR
+ *                                 from the start of each thread block (a launch of either takes well under 1 ms)
+ *   IPOT_TUNE_TEST_WITHHOLD_RANK  for tests of the give-up path only: CTA `value` (0-7) of every cluster
+ *                                 (IPOT_SCORER_TENSOR_SWEEPS) or of the grid (IPOT_SCORER_TENSOR) never reports its
+ *                                 statistics, so every wait for them runs into the limit; -1 = off (default)
  * Errors: INVALID (unknown `what`, value out of range).  Takes effect at the next launch.
  */
 enum {

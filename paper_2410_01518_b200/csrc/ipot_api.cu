@@ -273,7 +273,8 @@ int run_scoring(ipot *p, const void *Q, const void *Kc, int cap_rows, const floa
     if (scorer == IPOT_SCORER_TENSOR) {
         int n_launch = 0;
         rc = tc_launch(p->tc, p->cfg, Q, score_keys(p), cap_stats, p->scores, (size_t)p->units * p->cfg.pot_size, N, M, p->units, p->status,
-                       p->stream, parts, &n_launch, keys_in_chunk ? p->pend_K : nullptr, keys_in_chunk ? p->pend_first : 0);
+                       p->stream, parts, &n_launch, keys_in_chunk ? p->pend_K : nullptr, keys_in_chunk ? p->pend_first : 0, p->ts.wait_ns,
+                       p->ts.withhold_rank);
         p->launches += n_launch;
     } else if (scorer == IPOT_SCORER_TENSOR_SWEEPS) {
         rc = ts_launch(p->tc, p->ts_occ, p->ts, p->cfg, Q, score_keys(p), cap_stats, p->scores, N, M, p->units, p->status, p->stream,

@@ -37,9 +37,13 @@
 // Blocks of one grid wait on each other (pass 2 needs the other slabs' statistics),
 // so the grid is launched cooperatively with at most one CTA per SM: all of it is
 // resident.  A CTA publishes pass 1 of task t+1 before it waits for task t, so the
-// waits cannot form a cycle.  Every wait (mbarrier or statistics) is bounded; one that
-// runs out records IPOT_E_TIMEOUT in the status word and lets the CTA run to its
-// normal end with tensor memory released.
+// waits cannot form a cycle.  Every wait (mbarrier or statistics) is bounded by a time
+// limit (a launch parameter); one that runs out records IPOT_E_TIMEOUT in the status
+// word and raises a block-wide flag.  From then on every wait of the block returns at
+// once: the producer and the MMA issuer stop putting work in flight and wait for what
+// they have issued (loads into this CTA's shared memory, MMAs into its tensor memory)
+// before the block releases tensor memory and ends; the epilogue warps run through
+// their remaining iterations without waiting (their results are void).
 #pragma once
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -57,7 +61,6 @@ constexpr int kTcD = 128;            // largest head dimension; 64 uses the firs
 constexpr uint32_t kTcQBytes = kTcRows * kTcD * 2;           // 32 KiB: two halves of 128 rows x 64 channels
 constexpr uint32_t kTcKBytes = kTcSlab * kTcD * 2;           // 64 KiB: two halves of 256 rows x 64 channels
 constexpr uint32_t kTcStageBytes = kTcQBytes + kTcKBytes;    // 96 KiB
-constexpr uint32_t kTcSpinLimit = 1u << 22;                  // try_wait / poll rounds before giving up
 
 // shared-memory carve-up (bytes from the 1024-aligned base)
 constexpr uint32_t kTcOffStage = 0;                                        // [2] { Q, K }
@@ -65,12 +68,12 @@ constexpr uint32_t kTcOffColpart = 2 * kTcStageBytes;                      // [2
 constexpr uint32_t kTcOffTstat = kTcOffColpart + 2 * 4 * kTcSlab * 4;          // [2 buffers][8 chunks][128] float2
 constexpr uint32_t kTcOffFbuf = kTcOffTstat + 2 * 8 * kTcRows * 8;         // [2 buffers][8 chunks][128] float
 constexpr uint32_t kTcOffBar = kTcOffFbuf + 2 * 8 * kTcRows * 4;
-constexpr uint32_t kTcOffTmemSlot = kTcOffBar + 128;                       // the allocated TMEM base address
-constexpr uint32_t kTcOffAbort = kTcOffBar + 132;                          // set once a wait of the CTA has run out
+constexpr uint32_t kTcOffTmemSlot = kTcOffBar + 192;                       // the allocated TMEM base address
+constexpr uint32_t kTcOffAbort = kTcOffBar + 196;                          // set once a wait of the CTA has run out; + 4: the block's deadline (8 bytes)
 constexpr uint32_t kTcSmemBytes = kTcOffBar + 256;                         // no static shared memory: the base is 1024-aligned
 
 // barriers: per stage Full, Empty, EReady, FReady; per (buffer, half) SFull, TEmpty at index 2 * buffer + half
-enum { kBarFull = 0, kBarEmpty = 2, kBarEReady = 4, kBarFReady = 6, kBarSFull = 8, kBarTEmpty = 12, kBarCount = 16 };
+enum { kBarFull = 0, kBarEmpty = 2, kBarEReady = 4, kBarFReady = 6, kBarSFull = 8, kBarTEmpty = 12, kBarDrain = 16, kBarCount = 17 };
 
 struct TcParams {
     float *scores;        // partial array p (query rows 128p ...) at scores + p * part_stride, unit stride N
@@ -78,6 +81,8 @@ struct TcParams {
     float2 *stats;        // [items][slabs][128] (max in log2 units, sum * sign); all of the other sign or 0 at launch
     const float2 *cap_stats;  // NULL, or [units][M] (max, sum) over the CaP's own keys that join every row's denominator
     float sign;           // +1 or -1: this launch's "fresh" mark
+    unsigned long long wait_ns;  // limit of every wait
+    int withhold_cta;     // -1; test hook: this CTA never publishes its slab statistics
     int *status;
     int N, M, mtiles, slabs, tasks;
     int dhalves;          // d / 64: 64-channel halves of a tile (1 or 2)
@@ -111,15 +116,30 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait.  Once any wait of the CTA has run out, later waits return at once.
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status)
+__device__ __forceinline__ unsigned long long global_ns()
 {
-    for (uint32_t i = 0; i < kTcSpinLimit; ++i) {
-        if (mbar_try_wait(bar, parity)) return;
-        if ((i & 1023u) == 1023u && *abort_flag) return;
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait.  Every block notes a deadline (its start + the launch's wait limit) next to its give-up flag; a
+// wait that is still unsatisfied then records IPOT_E_TIMEOUT and raises the flag.  Once the flag is up, later waits
+// of the block return at once (false) - unless heed_flag is off, which is how a role waits for work it has itself
+// put in flight before the block may end.  (Clock and flag are looked at every 1024 rounds only: the kernel's
+// speed depends on this loop staying small.)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, bool heed_flag = true)
+{
+    for (uint32_t i = 0;; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 1023u) == 1023u) {
+            if (heed_flag && *abort_flag) return false;
+            if (global_ns() > *reinterpret_cast<volatile unsigned long long *>(abort_flag + 1)) {
+                *abort_flag = 1;
+                set_status(status, kStatusTimeout);
+                return false;
+            }
+        }
     }
-    *abort_flag = 1;
-    set_status(status, kStatusTimeout);
 }
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int c0, int c1, int c2, uint32_t bar)
@@ -361,6 +381,7 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
+        *reinterpret_cast<unsigned long long *>(gbase + kTcOffAbort + 4) = global_ns() + prm.wait_ns;
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar(kBarFull + b), 1);
             mbar_init(bar(kBarEmpty + b), 1);
@@ -371,6 +392,7 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                 mbar_init(bar(kBarTEmpty + 2 * b + h), 512);
             }
         }
+        mbar_init(bar(kBarDrain), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {  // tensor memory: two buffers of 256 columns
@@ -392,7 +414,7 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                 const int item = task / tasks_per_item, slab = task - item * tasks_per_item;
                 const int unit = item / prm.mtiles, mt = item - unit * prm.mtiles;
                 const uint32_t b = k & 1, ph = (k >> 1) & 1;
-                mbar_wait(bar(kBarEmpty + b), ph ^ 1, ab, prm.status);
+                if (!mbar_wait(bar(kBarEmpty + b), ph ^ 1, ab, prm.status)) break;   // nothing more is put in flight
                 mbar_expect_tx(bar(kBarFull + b), (uint32_t)prm.dhalves * (kTcStageBytes / 2));
                 const uint32_t q = base + kTcOffStage + b * kTcStageBytes, kk = q + kTcQBytes;
                 const bool fresh_rows = slab >= prm.new_slab0;
@@ -405,6 +427,10 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                     tma_load_3d(kk + kTcKBytes / 2, mk, 64, krow, unit, bar(kBarFull + b));
                 }
             }
+            // loads that were issued land in this CTA's shared memory: see the last one of either stage complete before
+            // the CTA may end (k loads were issued; load j went to stage j & 1 as its (j >> 1)-th fill)
+            for (uint32_t j = (k > 2 ? k - 2 : 0); j < k; ++j)
+                mbar_wait(bar(kBarFull + (j & 1)), (j >> 1) & 1, ab, prm.status, false);
         }
         __syncwarp();
     } else if (warp == 1) {
@@ -413,10 +439,10 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
             uint32_t k = 0;
             for (int task = blockIdx.x; task < prm.tasks; task += gridDim.x, ++k) {
                 const uint32_t b = k & 1, ph = (k >> 1) & 1;
-                mbar_wait(bar(kBarFull + b), ph, ab, prm.status);
+                if (!mbar_wait(bar(kBarFull + b), ph, ab, prm.status)) break;
                 const uint32_t qa = base + kTcOffStage + b * kTcStageBytes, kb = qa + kTcQBytes;
                 for (uint32_t h = 0; h < 2; ++h) {
-                    mbar_wait(bar(kBarTEmpty + 2 * b + h), ph ^ 1, ab, prm.status);
+                    if (!mbar_wait(bar(kBarTEmpty + 2 * b + h), ph ^ 1, ab, prm.status)) break;
                     tc_fence_after();
                     for (uint32_t blk = 0; blk < (uint32_t)prm.dhalves; ++blk) {
 #pragma unroll
@@ -429,7 +455,12 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                     }
                     tc_commit(bar(kBarSFull + 2 * b + h));   // this half's logits are complete
                 }
+                if (*ab) break;
                 tc_commit(bar(kBarEmpty + b));               // the stage may be refilled once the MMAs have read it
+            }
+            if (k) {  // every MMA has finished (and read its operands) before tensor memory is released
+                tc_commit(bar(kBarDrain));
+                mbar_wait(bar(kBarDrain), 0, ab, prm.status, false);
             }
         }
         __syncwarp();
@@ -541,7 +572,7 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
             }
             const float ms = max3(max3(cm[0], cm[1], cm[2]), max3(cm[3], cm[4], cm[5]), fmaxf(cm[6], cm[7]));
             const float ls = ((ce[0] + ce[1]) + (ce[2] + ce[3])) + ((ce[4] + ce[5]) + (ce[6] + ce[7]));
-            if (tasks_per_item > 1) st_gpu_f32x2(&prm.stats[((size_t)item * tasks_per_item + slab) * kTcRows + row], ms, ls * sgn);
+            if (tasks_per_item > 1 && (int)blockIdx.x != prm.withhold_cta) st_gpu_f32x2(&prm.stats[((size_t)item * tasks_per_item + slab) * kTcRows + row], ms, ls * sgn);
 
             // ---- this row's statistics of every slab of the item; re-read until all carry this launch's mark
             const float2 *st = prm.stats + (size_t)item * tasks_per_item * kTcRows + row;
@@ -564,7 +595,7 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                         if (!(sv[s].y * sgn > 0.f)) sv[s] = ld_gpu_f32x2(&st[(size_t)(s0 + s) * kTcRows]);
                         fresh = fresh && (sv[s].y * sgn > 0.f);
                     }
-                    if (!fresh && ((++tries > kTcSpinLimit) || *ab)) {
+                    if (!fresh && (*ab || ((++tries & 1023u) == 0 && global_ns() > *reinterpret_cast<volatile unsigned long long *>(ab + 1)))) {
                         if (!*ab) {
                             *ab = 1;
                             set_status(prm.status, kStatusTimeout);
@@ -692,7 +723,8 @@ inline int tc_encode_rows(TcPlan &plan, CUtensorMap *map, const void *ptr, int d
 // array (the chunk of a deferred append); new_first must be a multiple of the slab size.
 inline int tc_launch(TcPlan &plan, const ipot_config_t &cfg, const void *Q, const void *K, const float2 *cap_stats, float *scores,
                      size_t part_stride, int N, int M, int units, int *status, cudaStream_t stream, int *parts, int *n_launch,
-                     const void *Knew = nullptr, int new_first = 0)
+                     const void *Knew = nullptr, int new_first = 0, unsigned long long wait_ns = 200ull * 1000 * 1000,
+                     int withhold_cta = -1)
 {
     if (!tc_applicable(plan, cfg, N, M)) return IPOT_E_INVALID;
     if (Knew && (new_first % kTcSlab != 0 || new_first >= N)) return IPOT_E_INVALID;
@@ -715,6 +747,8 @@ inline int tc_launch(TcPlan &plan, const ipot_config_t &cfg, const void *Q, cons
     prm.dhalves = cfg.d / 64;
     prm.new_slab0 = Knew ? new_first / kTcSlab : 0x7fffffff;
     prm.scale_log2e = (float)(1.4426950408889634 / sqrt((double)cfg.d));
+    prm.wait_ns = wait_ns;
+    prm.withhold_cta = withhold_cta;
     if (items != plan.last_items || prm.slabs != plan.last_slabs) {
         if (cudaMemsetAsync(plan.stats, 0, (size_t)items * prm.slabs * kTcRows * sizeof(float2), stream) != cudaSuccess) {
             cudaGetLastError();

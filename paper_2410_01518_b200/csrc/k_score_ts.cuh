@@ -136,12 +136,6 @@ __device__ __forceinline__ float2 ld_cluster_f32x2(uint32_t cluster_addr)
     asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(cluster_addr) : "memory");
     return v;
 }
-__device__ __forceinline__ unsigned long long global_ns()
-{
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
 __device__ __forceinline__ float lg2(float x)
 {
     float y;

@@ -119,16 +119,18 @@ def test_sweeps_refuses_shapes_it_does_not_take():
             ipot.ipot_destroy(h)
 
 
-def test_a_wait_that_runs_out_ends_the_launch_with_a_status_and_the_pot_recovers():
-    """One CTA of every cluster never reports its row statistics (a test hook: nothing is damaged, the others' wait for
-    them simply cannot end) and the wait limit is 2 ms: the launch must end by itself, the status word must say
-    IPOT_E_TIMEOUT, and after ipot_reset the same pot must run a correct cycle with the hook off."""
+@pytest.mark.parametrize("scorer", [SW, ipot.IPOT_SCORER_TENSOR])
+def test_a_wait_that_runs_out_ends_the_launch_with_a_status_and_the_pot_recovers(scorer):
+    """One CTA (of every cluster, or of the one-sweep kernel's grid) never reports its statistics (a test hook: nothing
+    is damaged, the others' wait for them simply cannot end) and the wait limit is 2 ms: the launch must end by
+    itself, the status word must say IPOT_E_TIMEOUT, and after ipot_reset the same pot must run a correct cycle with
+    the hook off."""
     cfg = inputs.small_config(cfg_id=483, pot_size=1024, keep=400, nuc_slots=100, cap_rows=16, Hq=8, Hkv=2, d=128,
                               dtype="bf16", layers=2)
     t = inputs.make_cycle(cfg)
     h = make_pot(cfg)
     try:
-        ipot.ipot_set_scorer(h, SW)
+        ipot.ipot_set_scorer(h, scorer)
         ipot.ipot_set_tuning(h, ipot.IPOT_TUNE_SWEEPS_CLUSTER, 2)
         ipot.ipot_set_tuning(h, ipot.IPOT_TUNE_WAIT_LIMIT_NS, 2_000_000)
         ipot.ipot_set_tuning(h, ipot.IPOT_TUNE_TEST_WITHHOLD_RANK, 1)
