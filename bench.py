@@ -35,6 +35,10 @@ REFERENCE_BUDGET_S = 150.0   # wall-clock budget of a whole --impl reference run
 NOVELTY_WORKLOADS = {"nuc32k": (32000, 2048), "nuc128k": (128256, 2048)}
 # generation over a full pot alone: one new token's attention over all layers' units, configs[cfg - 1] shape
 DECODE_WORKLOADS = {"decode3": 3, "decode4": 4, "decode5": 5}
+SCORERS = {"auto": 0, "simt": 1, "tensor": 2, "warp_mma": 3, "sweeps": 4}
+SCORER_KERNELS = {1: "cap_row_stats + cap_column_sums (fp32 FMA)", 2: "cap_score_tc_kernel (tcgen05, one sweep)",
+                  3: "cap_row_stats_mma + cap_column_sums_mma (mma.sync)", 4: "cap_score_ts_kernel (tcgen05, two sweeps)"}
+MIN_SAMPLED_S = 1.0   # the clock sampler should see at least this much of timed running
 RING = 4  # distinct chunks / query sets cycled through
 PREHEAT_S = 0.5  # untimed running before the warm-up steps, see main()
 
@@ -46,6 +50,18 @@ def peaks():
         return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
                 "source": "measured"}
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1400.0, "source": "fallback"}
+
+
+def recorded_traffic(kernel: str, shape: str, units: int):
+    """dram__bytes_read + dram__bytes_write of one launch, scaled to `units` from the capture on record."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.txt")
+    if not os.path.exists(path):
+        return None
+    for row in open(path):
+        f = row.split()
+        if len(f) >= 4 and not row.startswith("#") and f[0] == kernel and f[1] == shape:
+            return float(f[3]) * units / float(f[2])
+    return None
 
 
 def workload_shape(cfg):
@@ -267,7 +283,7 @@ def run_decode(args):
                             dtype=ipot.IPOT_BF16 if cfg.dtype == "bf16" else ipot.IPOT_F32, nuc_slots=cfg.nuc_slots, max_cap_rows=1)
     stream = torch.cuda.current_stream()
     ipot.ipot_set_stream(h, stream.cuda_stream)
-    ipot.ipot_set_scorer(h, {"auto": 0, "simt": 1, "tensor": 2}[args.scorer])
+    ipot.ipot_set_scorer(h, SCORERS[args.scorer])
     tensor_path = args.scorer != "simt" and cfg.dtype == "bf16" and cfg.d in (64, 128)
     K, V = inputs.make_kv(cfg, N)
     ipot.ipot_append_chunk(h, dev(K), dev(V), N)
@@ -477,7 +493,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg3", choices=sorted(WORKLOADS) + sorted(NOVELTY_WORKLOADS) + sorted(DECODE_WORKLOADS))
-    ap.add_argument("--scorer", default="auto", choices=["auto", "simt", "tensor"])
+    ap.add_argument("--scorer", default="auto", choices=sorted(SCORERS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cap-keys", action="store_true",
                     help="score with the CaP's own keys inside the softmax (the Appendix B listing read literally)")
@@ -534,7 +550,7 @@ def main():
     h = ipot.ipot_create_ex(cfg.pot_size, cfg.keep, cfg.layers, cfg.Hq, cfg.Hkv, cfg.d, batch=cfg.batch,
                             dtype=ipot.IPOT_BF16 if cfg.dtype == "bf16" else ipot.IPOT_F32,
                             nuc_slots=cfg.nuc_slots, max_cap_rows=cfg.cap_rows)
-    ipot.ipot_set_scorer(h, {"auto": 0, "simt": 1, "tensor": 2}[args.scorer])
+    ipot.ipot_set_scorer(h, SCORERS[args.scorer])
     if args.rope:
         rope_tables = [dev(a) for a in inputs.make_rope_table(cfg.pot_size, cfg.d, cfg.dtype)]
         ipot.ipot_enable_rope(h, rope_tables[0], rope_tables[1], ipot.IPOT_ROPE_HALF)
@@ -569,22 +585,27 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    def timed(step, steps, warmup, sampler=None):
+    def timed(step, steps, warmup, sampler=None, repeats=1):
+        """Exactly `steps` steps between two events, bracketed by barrier + synchronize; with repeats > 1 the same
+        region is run that many times (each bracketed the same way) and the median region counts."""
         for i in range(warmup):
             step(i)
         barrier()
         if sampler:
             sampler.start()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         l0 = ipot.ipot_launch_count(h)
-        e0.record(stream)
-        for i in range(steps):
-            step(warmup + i)
-        e1.record(stream)
-        barrier()
+        times = []
+        for r in range(repeats):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for i in range(steps):
+                step(warmup + r * steps + i)
+            e1.record(stream)
+            barrier()
+            times.append(e0.elapsed_time(e1))
         clocks = sampler.stop() if sampler else None
-        rate, ms_step = whole_job_rate(e0.elapsed_time(e1), steps, world, "cuda")
-        return rate, ms_step, ipot.ipot_launch_count(h) - l0, clocks
+        rate, ms_step = whole_job_rate(float(np.median(times)), steps, world, "cuda")
+        return rate, ms_step, (ipot.ipot_launch_count(h) - l0) // repeats, clocks
 
     # untimed pre-heat: the first few hundred milliseconds after idle run at lower memory throughput (the compaction
     # kernel takes 105 us averaged over the first 0.1 s of steps, 91 us over 0.3 s, 82 us afterwards)
@@ -596,8 +617,15 @@ def main():
             i += 1
         torch.cuda.synchronize()
     # device-resident inputs: the headline value over exactly K steps, no instrumentation inside the region
+    # a short region (few steps) is repeated so that the clock sampler sees MIN_SAMPLED_S of it; the median region counts
+    _, ms_probe, _, _ = timed(step_dev, 20, 0)
+    repeats = int(min(2000, max(1, np.ceil(MIN_SAMPLED_S * 1e3 / (ms_probe * args.steps)))))
+    if world > 1:   # every rank must run the same number of regions
+        r_t = torch.tensor([repeats], device="cuda")
+        dist.all_reduce(r_t, op=dist.ReduceOp.MAX)
+        repeats = int(r_t.item())
     sampler = ClockSampler(local)
-    value, ms_step, launches, clocks = timed(step_dev, args.steps, args.warmup, sampler)
+    value, ms_step, launches, clocks = timed(step_dev, args.steps, args.warmup, sampler, repeats)
     assert ipot.ipot_sync_status(h) == 0, "device status is not clean"
     # the same K steps once more with the library's per-kernel CUDA events (they serialise the kernel boundaries,
     # which costs a few microseconds per step: reported beside the headline, not as it)
@@ -627,38 +655,56 @@ def main():
     pk = peaks()
     units, e, d, M = cfg.units, cfg.elem_bytes, cfg.d, cfg.G * cfg.cap_rows
     score_bytes = units * (N * d * e + M * d * e + 4 * N)      # K once + Q + scores out
-    score_flops = 2.0 * units * M * N * d
+    score_flops = 2.0 * units * M * N * d                      # one pass (a second sweep is overhead, not algorithm)
     # K and V, read + write, all kept rows; in rotary mode the rotated copy of K is written as well
     compact_bytes = units * (5 if args.rope else 4) * cfg.keep * d * e
     names = ["nuc_rank", "cap_score", "select", "compact"]
     # the dominant kernel; scoring and compaction are close, scoring is named unless compaction is clearly longer
     dom = 3 if kms[3] > 1.05 * kms[1] else 1
+    score_gbs = score_bytes / (kms[1] * 1e-3) / 1e9
+    score_tflops = score_flops / (kms[1] * 1e-3) / 1e12
     if names[dom] == "compact":
         roof = {"kernel": "compact_kernel", "bound": "hbm", "achieved": compact_bytes / (kms[3] * 1e-3) / 1e9,
                 "peak": pk["hbm_gbs"], "unit": "GB/s"}
     else:
-        roof = {"kernel": "cap_score (" + ("tcgen05" if scorer_used == 2 else "simt") + ")", "bound": "hbm",
-                "achieved": score_bytes / (kms[1] * 1e-3) / 1e9, "peak": pk["hbm_gbs"], "unit": "GB/s"}
+        # which roof binds Eq. 2 on this shape: reading K once at the copy rate, or 2 M N d flops per unit at the
+        # sustained bf16 rate (the fp32-FMA scorer is not a tensor-core kernel: its line is reported against HBM)
+        t_hbm = score_bytes / (pk["hbm_gbs"] * 1e9)
+        t_tensor = score_flops / (pk["bf16_tflops"] * 1e12) if cfg.dtype == "bf16" and scorer_used != 1 else 0.0
+        kernel = SCORER_KERNELS.get(scorer_used, "cap_score")
+        if t_tensor > t_hbm:
+            roof = {"kernel": kernel, "bound": "tensor", "achieved": score_tflops, "peak": pk["bf16_tflops"], "unit": "TFLOP/s"}
+        else:
+            roof = {"kernel": kernel, "bound": "hbm", "achieved": score_gbs, "peak": pk["hbm_gbs"], "unit": "GB/s"}
+        roof["roof_us"] = {"hbm": round(t_hbm * 1e6, 2), "tensor": round(t_tensor * 1e6, 2)}
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["peak_source"] = pk["source"]
-    roof["frac_of_nominal_8tbs"] = roof["achieved"] / 8000.0   # the HBM3e data-sheet figure, for context
-    # DRAM bytes of one launch of the scoring kernel from the committed ncu capture (profiles/): 71.198 MB for
-    # 64 units of this shape, growing with the units; unknown for other shapes, kernels or scorers
-    roof["traffic"] = (units * 71.198e6 / 64 if dom == 1 and scorer_used == 2 and (N, M, d) == (4096, 128, 128) and not args.cap_keys else None)
+    if roof["unit"] == "GB/s":
+        roof["frac_of_nominal_8tbs"] = roof["achieved"] / 8000.0   # the HBM3e data-sheet figure, for context
+    # DRAM bytes of one launch of the dominant kernel, from the committed ncu captures (profiles/dram_traffic.txt: measured
+    # on a few layers of the same shape and scaled by the units, which is how the traffic grows); null if no capture
+    # of this kernel and shape is on record
+    tkey = {1: "simt", 2: "cap_score_tc", 3: "warp_mma", 4: "cap_score_ts"}.get(scorer_used, "?") if dom == 1 else "compact"
+    roof["traffic"] = None if (args.cap_keys or args.rope) else recorded_traffic(tkey, f"N{N}_M{M}_d{d}_{cfg.dtype}", units)
     roof["kernel_ms"] = dict(zip(names, [round(x, 5) for x in kms]))
     roof["cycles_averaged"] = kcycles
-    roof["cap_score_gbs"] = score_bytes / (kms[1] * 1e-3) / 1e9
-    roof["cap_score_tflops"] = score_flops / (kms[1] * 1e-3) / 1e12
+    roof["cap_score_gbs"] = score_gbs
+    roof["cap_score_tflops"] = score_tflops
+    roof["cap_score_frac_of_hbm_peak"] = score_gbs / pk["hbm_gbs"]
+    roof["cap_score_frac_of_bf16_sustained"] = score_tflops / pk["bf16_tflops"]
     roof["compact_gbs"] = compact_bytes / (kms[3] * 1e-3) / 1e9
+    roof["compact_frac_of_hbm_peak"] = roof["compact_gbs"] / pk["hbm_gbs"]
 
     line = {
         "metric": "ccd_cycles_per_s", "value": value, "unit": "cycles/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
-        "config": dict(config_dict(cfg, n_new, N, args.cap_keys, getattr(args, "rope", False)), preheat_s=PREHEAT_S,
-                       append=("deferred: the chunk stays in the caller's device buffers, the scorer reads its keys there, "
-                               "the compaction copies the surviving rows into the pot" if args.append == "deferred"
-                               else "eager: all rows copied into the pot by the append call")),
+        "config": config_dict(cfg, n_new, N, args.cap_keys, getattr(args, "rope", False)),
+        "preheat_s": PREHEAT_S,   # untimed running before the warm-up steps: the value is a warm steady state
+        "append": ("deferred: the chunk stays in the caller's device buffers, the scorer reads its keys there, "
+                   "the compaction copies the surviving rows into the pot" if args.append == "deferred"
+                   else "eager: all rows copied into the pot by the append call"),
+        "repeats": repeats,       # timed regions of `steps` steps each; ms_per_step is the median region's
         "pot_tokens_per_s": value * N * cfg.batch,
         "layer_cycles_per_s": value * cfg.layers,
         "ms_per_step_with_kernel_events": ms_step_events,

@@ -76,6 +76,9 @@ struct ipot {
     TcPlan tc;           // tensor-core scorer state
     TsTuning ts;         // launch parameters of the two-sweep tensor-core scorer
     TsOccupancy ts_occ;
+    // the novelty ranking does not depend on the scores: it runs beside the scorer on a stream of its own
+    cudaStream_t side;
+    cudaEvent_t ev_fork, ev_join;
 };
 
 namespace {
@@ -117,6 +120,9 @@ void free_all(ipot *p)
     cudaFree(p->K); cudaFree(p->V); cudaFree(p->Krot); cudaFree(p->scores); cudaFree(p->summed);
     cudaFree(p->row_stats); cudaFree(p->mma_part); cudaFree(p->cap_stats); cudaFree(p->nuc_mask); cudaFree(p->idx); cudaFree(p->status);
     cudaFree(p->stage_q); cudaFree(p->stage_kc); cudaFree(p->stage_aux); cudaFree(p->nov_scratch); cudaFree(p->dec_partial); cudaFree(p->dec_counters);
+    if (p->ev_fork) cudaEventDestroy(p->ev_fork);
+    if (p->ev_join) cudaEventDestroy(p->ev_join);
+    if (p->side) cudaStreamDestroy(p->side);
     if (p->ev) {
         for (int i = 0; i < kProfSlots; ++i)
             for (auto &e : p->ev[i]) if (e) cudaEventDestroy(e);
@@ -257,10 +263,20 @@ int run_scoring(ipot *p, const void *Q, const void *Kc, int cap_rows, const floa
 
     cudaEvent_t *ev = (p->profiling && p->ev_used < kProfSlots) ? p->ev[p->ev_used] : nullptr;
     if (ev) IPOT_CUDA(cudaEventRecord(ev[0], p->stream));
+    // Sec. 3.3.3: the T most novel slots per stream.  One block per stream and independent of the scores, so it is
+    // queued on the side stream (after everything the caller has queued so far) and the tensor-core scorers leave
+    // it one SM; the selection waits for both.  Other scorers fill the device in waves and need no such care.
+    const bool side_nuc = T > 0 && aux && p->side && (scorer == IPOT_SCORER_TENSOR || scorer == IPOT_SCORER_TENSOR_SWEEPS);
     if (T > 0 && aux) {
-        nuc_mask_kernel<<<p->cfg.batch, kSelThreads, (size_t)N * 4, p->stream>>>(aux, p->nuc_mask, N, T);
+        cudaStream_t ns = side_nuc ? p->side : p->stream;
+        if (side_nuc) {
+            IPOT_CUDA(cudaEventRecord(p->ev_fork, p->stream));
+            IPOT_CUDA(cudaStreamWaitEvent(p->side, p->ev_fork, 0));
+        }
+        nuc_mask_kernel<<<p->cfg.batch, kSelThreads, (size_t)N * 4, ns>>>(aux, p->nuc_mask, N, T);
         p->launches += 1;
         IPOT_CUDA(cudaGetLastError());
+        if (side_nuc) IPOT_CUDA(cudaEventRecord(p->ev_join, p->side));
     }
     if (ev) IPOT_CUDA(cudaEventRecord(ev[1], p->stream));
     *parts = 1;
@@ -274,17 +290,18 @@ int run_scoring(ipot *p, const void *Q, const void *Kc, int cap_rows, const floa
         int n_launch = 0;
         rc = tc_launch(p->tc, p->cfg, Q, score_keys(p), cap_stats, p->scores, (size_t)p->units * p->cfg.pot_size, N, M, p->units, p->status,
                        p->stream, parts, &n_launch, keys_in_chunk ? p->pend_K : nullptr, keys_in_chunk ? p->pend_first : 0, p->ts.wait_ns,
-                       p->ts.withhold_rank);
+                       p->ts.withhold_rank, side_nuc ? 1 : 0);
         p->launches += n_launch;
     } else if (scorer == IPOT_SCORER_TENSOR_SWEEPS) {
         rc = ts_launch(p->tc, p->ts_occ, p->ts, p->cfg, Q, score_keys(p), cap_stats, p->scores, N, M, p->units, p->status, p->stream,
-                       keys_in_chunk ? p->pend_K : nullptr, keys_in_chunk ? p->pend_first : 0);
+                       keys_in_chunk ? p->pend_K : nullptr, keys_in_chunk ? p->pend_first : 0, side_nuc ? 1 : 0);
         p->launches += 1;
     } else if (scorer == IPOT_SCORER_WARP_MMA) {
         rc = launch_warp_mma(p, Q, cap_stats, M, N);
     } else {
         rc = p->cfg.dtype == IPOT_F32 ? launch_simt<float>(p, Q, cap_stats, M, N) : launch_simt<__nv_bfloat16>(p, Q, cap_stats, M, N);
     }
+    if (side_nuc) IPOT_CUDA(cudaStreamWaitEvent(p->stream, p->ev_join, 0));   // (also when the scorer refused: nothing is left behind on the side stream)
     if (rc != IPOT_OK) return rc;
     if (ev) IPOT_CUDA(cudaEventRecord(ev[2], p->stream));
     p->last_scorer = scorer;
@@ -563,6 +580,14 @@ int ipot_create_ex(const ipot_config_t *cfg, ipot_t **out)
          cudaFuncSetAttribute(nuc_mask_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 32768 * 4) == cudaSuccess &&
          cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 32768 * 4) == cudaSuccess;
     if (!ok) {
+        cudaGetLastError();
+        free_all(p);
+        delete p;
+        return IPOT_E_CUDA;
+    }
+    if (cudaStreamCreateWithFlags(&p->side, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&p->ev_join, cudaEventDisableTiming) != cudaSuccess) {
         cudaGetLastError();
         free_all(p);
         delete p;

@@ -724,7 +724,7 @@ inline int tc_encode_rows(TcPlan &plan, CUtensorMap *map, const void *ptr, int d
 inline int tc_launch(TcPlan &plan, const ipot_config_t &cfg, const void *Q, const void *K, const float2 *cap_stats, float *scores,
                      size_t part_stride, int N, int M, int units, int *status, cudaStream_t stream, int *parts, int *n_launch,
                      const void *Knew = nullptr, int new_first = 0, unsigned long long wait_ns = 200ull * 1000 * 1000,
-                     int withhold_cta = -1)
+                     int withhold_cta = -1, int spare_sms = 0)
 {
     if (!tc_applicable(plan, cfg, N, M)) return IPOT_E_INVALID;
     if (Knew && (new_first % kTcSlab != 0 || new_first >= N)) return IPOT_E_INVALID;
@@ -760,7 +760,9 @@ inline int tc_launch(TcPlan &plan, const ipot_config_t &cfg, const void *Q, cons
     plan.sign = -plan.sign;
     prm.sign = plan.sign;
     cudaLaunchConfig_t lc = {};
-    lc.gridDim = dim3(prm.tasks < plan.sm_count ? prm.tasks : plan.sm_count, 1, 1);
+    // spare_sms: SMs left to a small kernel of the same cycle that runs beside this one on another stream
+    const int ctas = plan.sm_count - spare_sms > 0 ? plan.sm_count - spare_sms : 1;
+    lc.gridDim = dim3(prm.tasks < ctas ? prm.tasks : ctas, 1, 1);
     lc.blockDim = dim3(kTcThreads, 1, 1);
     lc.dynamicSmemBytes = kTcSmemBytes;
     lc.stream = stream;

@@ -848,7 +848,7 @@ inline int ts_pick_cluster(const TsOccupancy &occ, int units, int slabs)
 // [units][N - new_first][d] array (the chunk of a deferred append); new_first must be a multiple of the slab size.
 inline int ts_launch(TcPlan &plan, TsOccupancy &occ, const TsTuning &tune, const ipot_config_t &cfg, const void *Q, const void *K, const float2 *cap_stats,
                      float *scores, int N, int M, int units, int *status, cudaStream_t stream, const void *Knew = nullptr,
-                     int new_first = 0)
+                     int new_first = 0, int spare_sms = 0)
 {
     if (!ts_applicable(plan, cfg, N, M)) return IPOT_E_INVALID;
     constexpr int SK = kTsSlab;
@@ -878,7 +878,11 @@ inline int ts_launch(TcPlan &plan, TsOccupancy &occ, const TsTuning &tune, const
     if (cluster < 1 || occ.clusters[ci] < 1) return IPOT_E_CUDA;   // not even one such cluster fits this device
     cudaLaunchConfig_t lc;
     cudaLaunchAttribute at[1];
-    ts_launch_config(lc, at, cluster, units < occ.clusters[ci] ? units : occ.clusters[ci], stream);
+    // spare_sms: SMs left to a small kernel of the same cycle that runs beside this one on another stream
+    int clusters = occ.clusters[ci];
+    if (clusters * cluster > plan.sm_count - spare_sms) clusters = (plan.sm_count - spare_sms) / cluster;
+    if (clusters < 1) clusters = 1;
+    ts_launch_config(lc, at, cluster, units < clusters ? units : clusters, stream);
     void *args[4] = {(void *)&mapQ, (void *)&mapK, (void *)&mapKnew, (void *)&prm};
     if (cudaLaunchKernelExC(&lc, ts_kernel_ptr(tune.poly >= 0 ? tune.poly : kTsDefaultPoly), args) != cudaSuccess) {
         cudaGetLastError();
