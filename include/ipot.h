@@ -26,7 +26,10 @@
  *     only read.  Work is queued on the pot's stream and the call returns
  *     without waiting; the caller must keep the buffers alive and unchanged
  *     until that work has run (synchronise the stream or call
- *     ipot_sync_status()).
+ *     ipot_sync_status()).  Inside a cycle the library may run a kernel on a
+ *     stream of its own beside the others; it is forked from and joined back
+ *     into the pot's stream by events within the same call, so everything a
+ *     call has queued is ordered in the pot's stream when the call returns.
  *   - The library owns the pot, the score/index arrays and its scratch; they
  *     are allocated in ipot_create*() and freed in ipot_destroy().
  *   - A pot object is not thread-safe; use one host thread per pot at a time.
