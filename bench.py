@@ -694,6 +694,11 @@ def main():
     roof["cap_score_frac_of_bf16_sustained"] = score_tflops / pk["bf16_tflops"]
     roof["compact_gbs"] = compact_bytes / (kms[3] * 1e-3) / 1e9
     roof["compact_frac_of_hbm_peak"] = roof["compact_gbs"] / pk["hbm_gbs"]
+    # the whole step against the copy rate: algorithmic bytes of scoring + compaction (+ the append's copy when it is
+    # made at append time) over the step's time
+    step_bytes = score_bytes + compact_bytes + (0 if args.append == "deferred" else units * 4 * n_new * d * e)
+    roof["step_gbs"] = step_bytes / (ms_step * 1e-3) / 1e9
+    roof["step_frac_of_hbm_peak"] = roof["step_gbs"] / pk["hbm_gbs"]
 
     line = {
         "metric": "ccd_cycles_per_s", "value": value, "unit": "cycles/s", "n_gpus": world, "steps": args.steps,
