@@ -156,33 +156,6 @@ __device__ __forceinline__ float2 fadd2_ftz(float2 a, float2 b)
 }
 
 // ------------------------------------------------------------------ exponentials
-// 2^t for a pair, t <= 8, on the FMA pipe.  t is clamped at -126: with j = round(t) >= -126 and the polynomial in
-// [0.707, 1.415] the exponent field of the result stays >= 0.  Results below 2^-126 (the clamp included: the
-// polynomial is just below 1 at f = 0) come out as subnormal bit patterns; callers add them with flush-to-zero
-// arithmetic or against sums that hold a far larger term, which matches the special-function unit's zero.
-__device__ __forceinline__ float2 exp2_fma_pair(float2 t)
-{
-    t.x = fmaxf(t.x, -126.f);
-    t.y = fmaxf(t.y, -126.f);
-    const float2 magic = make_float2(12582912.f, 12582912.f);       // 1.5 * 2^23: adding it rounds t to an integer
-    const float2 r = __fadd2_rn(t, magic);
-    const float2 jf = __fadd2_rn(r, make_float2(-12582912.f, -12582912.f));
-    const float2 f = __ffma2_rn(jf, make_float2(-1.f, -1.f), t);    // in [-0.5, 0.5]
-    float2 p = __ffma2_rn(make_float2(0.009570101276f, 0.009570101276f), f, make_float2(0.05591785908f, 0.05591785908f));
-    p = __ffma2_rn(p, f, make_float2(0.2402474433f, 0.2402474433f));
-    p = __ffma2_rn(p, f, make_float2(0.6931217909f, 0.6931217909f));
-    p = __ffma2_rn(p, f, make_float2(0.9999992847f, 0.9999992847f));
-    // the integer sits in the low mantissa bits of r; the shift drops the rest of r
-    return make_float2(__int_as_float(__float_as_int(p.x) + (__float_as_int(r.x) << 23)),
-                       __int_as_float(__float_as_int(p.y) + (__float_as_int(r.y) << 23)));
-}
-// Pair i of a piece goes to the FMA pipe if its position in an evenly spread order of 8 is below kPoly.
-template <int kPoly>
-__device__ __forceinline__ constexpr bool pair_on_fma(int i)
-{
-    constexpr int order[8] = {0, 4, 2, 6, 1, 5, 3, 7};
-    return order[i & 7] < kPoly;
-}
 // (called from fully unrolled loops: the choice is a constant by the time code is generated)
 __device__ __forceinline__ float2 exp2_pair(bool on_fma, float2 t)
 {
