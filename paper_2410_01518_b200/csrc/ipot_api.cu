@@ -273,7 +273,7 @@ int run_scoring(ipot *p, const void *Q, const void *Kc, int cap_rows, const floa
             IPOT_CUDA(cudaEventRecord(p->ev_fork, p->stream));
             IPOT_CUDA(cudaStreamWaitEvent(p->side, p->ev_fork, 0));
         }
-        nuc_mask_kernel<<<p->cfg.batch, kSelThreads, (size_t)N * 4, ns>>>(aux, p->nuc_mask, N, T);
+        launch_nuc_mask(p->cfg.batch, ns, aux, p->nuc_mask, N, T);
         p->launches += 1;
         IPOT_CUDA(cudaGetLastError());
         if (side_nuc) IPOT_CUDA(cudaEventRecord(p->ev_join, p->side));
@@ -388,9 +388,8 @@ int run_cycle(ipot *p, const void *Q, const void *Kc, int cap_rows, const float 
     int rc = run_scoring(p, Q, Kc, cap_rows, aux, &parts);
     if (rc != IPOT_OK) return rc;
     const size_t part_stride = (size_t)p->units * p->cfg.pot_size;
-    select_kernel<<<p->units, kSelThreads, (size_t)N * 4, p->stream>>>(
-        p->scores, parts, part_stride, T > 0 ? p->nuc_mask : nullptr, p->idx,
-        parts > 1 ? p->summed : nullptr, N, keep, p->cfg.Hkv, p->cfg.batch, p->status);
+    launch_select(p->units, p->stream, p->scores, parts, part_stride, T > 0 ? p->nuc_mask : nullptr, p->idx,
+                  parts > 1 ? p->summed : nullptr, N, keep, p->cfg.Hkv, p->cfg.batch, p->status);
     p->launches += 1;
     IPOT_CUDA(cudaGetLastError());
     if (ev) IPOT_CUDA(cudaEventRecord(ev[3], p->stream));
@@ -576,9 +575,7 @@ int ipot_create_ex(const ipot_config_t *cfg, ipot_t **out)
          cudaFuncSetAttribute(cap_column_sums<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)simt_smem_bytes(256)) == cudaSuccess &&
          cudaFuncSetAttribute(cap_self_stats_bf16, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)self_smem_bytes(256)) == cudaSuccess &&
          cudaFuncSetAttribute(cap_row_stats_mma, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mma_scorer_smem_bytes(256)) == cudaSuccess &&
-         cudaFuncSetAttribute(cap_column_sums_mma, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mma_scorer_smem_bytes(256)) == cudaSuccess &&
-         cudaFuncSetAttribute(nuc_mask_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 32768 * 4) == cudaSuccess &&
-         cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 32768 * 4) == cudaSuccess;
+         cudaFuncSetAttribute(cap_column_sums_mma, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mma_scorer_smem_bytes(256)) == cudaSuccess;
     if (!ok) {
         cudaGetLastError();
         free_all(p);
