@@ -230,6 +230,23 @@ def test_exact_ties_resolve_to_lower_slots():
     assert same == n
 
 
+@pytest.mark.parametrize("pot,keep,T", [(4096, 2048, 1024), (9000, 5001, 100), (16400, 5000, 0), (20000, 12288, 4096)])
+def test_exact_ties_in_large_pots(pot, keep, T):
+    """Every score equal and every novelty equal: the survivors are the first `keep` slots whatever the pot size.
+    The sizes take the ranking kernels through each block shape (256, 512, 1024 threads; 16 and 32 slots a thread),
+    pots that are not a multiple of 16 slots, index lists of more than one output round and of odd length."""
+    cfg = inputs.small_config(cfg_id=231, pot_size=pot, keep=keep, nuc_slots=T, cap_rows=2, Hq=2, Hkv=2, d=32, dtype="f32")
+    t = inputs.make_cycle(cfg)
+    t["K"][:] = t["K"][:, :, :, :1, :]
+    t["aux"][:] = 0.25
+    u, idx, K, V = gpu_cycle(cfg, t)
+    for unit in range(cfg.units):
+        assert np.array_equal(idx[unit], np.arange(keep))
+        assert np.unique(u[unit]).size == 1
+    same, n = compare_cycle(cfg, t, (u, idx, K, V))
+    assert same == n
+
+
 def test_duplicated_tokens_and_heavy_tails():
     cfg = inputs.small_config(cfg_id=5, recipe="student_dup", dtype="bf16", pot_size=1200, keep=300,
                               nuc_slots=150, cap_rows=8, batch=2, Hq=8, Hkv=2, d=128)
