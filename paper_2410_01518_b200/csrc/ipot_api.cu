@@ -398,9 +398,18 @@ int run_cycle(ipot *p, const void *Q, const void *Kc, int cap_rows, const float 
     const int slices = p->compact_slices;
     const size_t unit_vecs = (size_t)p->cfg.pot_size * row_vecs;
     if (!p->rope) {
-        dim3 grid(slices, p->units, 2);
-        compact_kernel<<<grid, kMoveThreads, 0, p->stream>>>((uint4 *)p->K, (uint4 *)p->V, p->idx, keep, N, row_vecs,
-                                                            row_vecs / slices, unit_vecs, p->status, pending_rows(p));
+        // programmatic dependent launch: the grid is set up while the selection still runs and waits inside the kernel
+        cudaLaunchConfig_t lc = {};
+        lc.gridDim = dim3(slices, p->units, 2);
+        lc.blockDim = dim3(kMoveThreads, 1, 1);
+        lc.stream = p->stream;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at[0].val.programmaticStreamSerializationAllowed = 1;
+        lc.attrs = at;
+        lc.numAttrs = 1;
+        IPOT_CUDA(cudaLaunchKernelEx(&lc, compact_kernel, (uint4 *)p->K, (uint4 *)p->V, (const int32_t *)p->idx, keep, N, row_vecs,
+                                     row_vecs / slices, unit_vecs, p->status, pending_rows(p)));
         p->launches += 1;
     } else {
         launch_compact_rope(p, keep, N, row_vecs, unit_vecs);

@@ -97,6 +97,9 @@ compact_kernel(uint4 *__restrict__ potK, uint4 *__restrict__ potV, const int32_t
                int keep, int N, int row_vecs, int slice_vecs, size_t unit_vecs, int *status, PendingRows pend)
 {
     uint4 *base = (blockIdx.z ? potV : potK) + (size_t)blockIdx.y * unit_vecs + (size_t)blockIdx.x * slice_vecs;
+    // launched as a programmatic dependent of the selection: the blocks may be resident before it has ended and
+    // wait here for its index lists (returns at once after an ordinary launch)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const uint4 *alt = blockIdx.z ? pend.V : pend.K;
     if (alt) alt += (size_t)blockIdx.y * pend.unit_vecs + (size_t)blockIdx.x * slice_vecs;
     compact_body(base, idx + (size_t)blockIdx.y * keep, keep, N, row_vecs, slice_vecs, status, alt, alt ? pend.first : 0x7fffffff);

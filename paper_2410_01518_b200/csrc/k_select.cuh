@@ -234,6 +234,8 @@ select_kernel(const float *__restrict__ scores, int parts, size_t part_stride,
     const float *u = scores + (size_t)unit * N;
     const uint8_t *m = mask ? mask + (size_t)b * N : nullptr;
     const int slot0 = threadIdx.x * kKpt;
+    // the compaction may be made resident now; it waits for this grid's end before it reads an index
+    asm volatile("griddepcontrol.launch_dependents;");
     if (threadIdx.x < 256) sh.hist[threadIdx.x] = 0;
     uint32_t key[kKpt];
     // a reserved slot outranks every score: finite scores map below 0xFF800000
