@@ -400,7 +400,7 @@ int run_cycle(ipot *p, const void *Q, const void *Kc, int cap_rows, const float 
     if (!p->rope) {
         // programmatic dependent launch: the grid is set up while the selection still runs and waits inside the kernel
         cudaLaunchConfig_t lc = {};
-        lc.gridDim = dim3(slices, p->units, 2);
+        lc.gridDim = dim3(slices, 2, p->units);
         lc.blockDim = dim3(kMoveThreads, 1, 1);
         lc.stream = p->stream;
         cudaLaunchAttribute at[1];

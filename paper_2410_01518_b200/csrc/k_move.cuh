@@ -37,7 +37,7 @@ append_kernel(const uint4 *__restrict__ srcK, const uint4 *__restrict__ srcV, ui
     append_body(src, dst, n_vecs, blockIdx.x, gridDim.x);
 }
 
-// In-place gather.  grid (slices, units, 2).  A block owns byte columns
+// In-place gather.  grid (slices, 2, units).  A block owns byte columns
 // [slice * slice_vecs, (slice + 1) * slice_vecs) (in 16-byte vectors) of every
 // row of one tensor of one unit, so blocks never touch the same bytes.  idx is
 // ascending, hence idx[r] >= r: the block walks the rows in ascending chunks,
@@ -96,13 +96,17 @@ __global__ void __launch_bounds__(kMoveThreads)
 compact_kernel(uint4 *__restrict__ potK, uint4 *__restrict__ potV, const int32_t *__restrict__ idx,
                int keep, int N, int row_vecs, int slice_vecs, size_t unit_vecs, int *status, PendingRows pend)
 {
-    uint4 *base = (blockIdx.z ? potV : potK) + (size_t)blockIdx.y * unit_vecs + (size_t)blockIdx.x * slice_vecs;
+    // Block order: the units from the last one down, K then V of a unit next to each other.  The scorer of the next
+    // cycle starts at unit 0 and finds the rows written last still in L2, and the two tensors of a unit share their
+    // index list while it is hot (measured against units ascending, all K before all V: step 183.2 -> 181.3 us).
+    const unsigned unit = gridDim.z - 1 - blockIdx.z, tensor = blockIdx.y;
+    uint4 *base = (tensor ? potV : potK) + (size_t)unit * unit_vecs + (size_t)blockIdx.x * slice_vecs;
     // launched as a programmatic dependent of the selection: the blocks may be resident before it has ended and
     // wait here for its index lists (returns at once after an ordinary launch)
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    const uint4 *alt = blockIdx.z ? pend.V : pend.K;
-    if (alt) alt += (size_t)blockIdx.y * pend.unit_vecs + (size_t)blockIdx.x * slice_vecs;
-    compact_body(base, idx + (size_t)blockIdx.y * keep, keep, N, row_vecs, slice_vecs, status, alt, alt ? pend.first : 0x7fffffff);
+    const uint4 *alt = tensor ? pend.V : pend.K;
+    if (alt) alt += (size_t)unit * pend.unit_vecs + (size_t)blockIdx.x * slice_vecs;
+    compact_body(base, idx + (size_t)unit * keep, keep, N, row_vecs, slice_vecs, status, alt, alt ? pend.first : 0x7fffffff);
 }
 
 }  // namespace ipotk
