@@ -301,9 +301,9 @@ int run_scoring(ipot *p, const void *Q, const void *Kc, int cap_rows, const floa
     } else {
         rc = p->cfg.dtype == IPOT_F32 ? launch_simt<float>(p, Q, cap_stats, M, N) : launch_simt<__nv_bfloat16>(p, Q, cap_stats, M, N);
     }
+    if (ev && rc == IPOT_OK) IPOT_CUDA(cudaEventRecord(ev[2], p->stream));   // the scorer's end, before the join below
     if (side_nuc) IPOT_CUDA(cudaStreamWaitEvent(p->stream, p->ev_join, 0));   // (also when the scorer refused: nothing is left behind on the side stream)
     if (rc != IPOT_OK) return rc;
-    if (ev) IPOT_CUDA(cudaEventRecord(ev[2], p->stream));
     p->last_scorer = scorer;
     p->last_len_before = N;
     p->last_scores = (*parts > 1) ? p->summed : p->scores;
