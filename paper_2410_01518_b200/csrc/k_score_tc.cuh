@@ -222,6 +222,25 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32
           "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31]),
           "r"(taddr) : "memory");
 }
+// 16 consecutive fp32 columns of this thread's TMEM lane (asynchronous: see tmem_wait_ld16).
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15};"
+        ::"r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]),
+          "r"(taddr) : "memory");
+}
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 // Named barrier of the four epilogue warps (one per TMEM lane quarter) that own the same columns.
@@ -319,6 +338,29 @@ __device__ __forceinline__ float2 pass1_chunk(uint32_t taddr, int col0, int nval
     return make_float2((mxr == -INFINITY) ? -INFINITY : mxc, (s01.x + s01.y) + (s23.x + s23.y));
 }
 
+// The same over 16 columns of a full chunk: maximum into four running maxima / exponentials into four packed sums.
+// `first_pair`: index of the piece's first column pair within its chunk (it fixes which pairs take the FMA pipe).
+__device__ __forceinline__ void piece_max(const uint32_t (&v)[16], float (&mx)[4])
+{
+#pragma unroll
+    for (int i = 0; i < 16; i += 8) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) mx[j] = max3(mx[j], __uint_as_float(v[i + 2 * j]), __uint_as_float(v[i + 2 * j + 1]));
+    }
+}
+template <int kFirstPair>
+__device__ __forceinline__ void piece_exp(uint32_t (&v)[16], float c, float mxc, float2 (&sum)[4])
+{
+    const float2 c2 = make_float2(c, c), nm2 = make_float2(-mxc, -mxc);
+#pragma unroll
+    for (int i = 0; i < 16; i += 2) {
+        const float2 x = __ffma2_rn(make_float2(__uint_as_float(v[i]), __uint_as_float(v[i + 1])), c2, nm2);
+        const float2 e2 = pair_on_fma<kTcFmaEighths>(kFirstPair + (i >> 1)) ? exp2_fma_pair(x) : make_float2(ex2(x.x), ex2(x.y));
+        sum[(i >> 1) & 3] = __fadd2_rn(sum[(i >> 1) & 3], e2);
+        v[i] = __float_as_uint(e2.x);
+        v[i + 1] = __float_as_uint(e2.y);
+    }
+}
 // Pass 2 for one warp over 32 rows x 32 columns: a[] and b[] are the 16x256b loads of the warp's TMEM lanes
 // 0..15 and 16..31, fr2[i] the weight of row lane/4 + 8i duplicated into both halves.  On exit
 // x[2j + h] = sum over this thread's four rows of f_r e[r][8j + 2(lane%4) + h].
@@ -487,13 +529,48 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                 const int nvalid = min(kTcSlab, prm.N - slab * kTcSlab);
                 const uint32_t b = k & 1, ph = (k >> 1) & 1;
                 const uint32_t t0 = tmem + ((uint32_t)(q * 32) << 16) + b * kTcSlab + cq * 32;
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    mbar_wait(bar(kBarSFull + 2 * b + h), ph, ab, prm.status);
+                if (nvalid == kTcSlab) {
+                    // two chunks of 32 columns (one per buffer half) in four pieces of 16 through two register sets:
+                    // the second half's first piece is fetched while the first half's second piece is still being
+                    // exponentiated, so that its tensor-memory latency is not waited for
+                    uint32_t X[16], Y[16];
+                    mbar_wait(bar(kBarSFull + 2 * b), ph, ab, prm.status);
                     tc_fence_after();
-                    const float2 st = (nvalid == kTcSlab) ? pass1_chunk<true>(t0 + h * 128, h * 128 + cq * 32, nvalid, c)
-                                                          : pass1_chunk<false>(t0 + h * 128, h * 128 + cq * 32, nvalid, c);
-                    tstat[(b * 8 + h * 4 + cq) * kTcRows + row] = st;
+                    tmem_ld16(t0, X);
+                    tmem_ld16(t0 + 16, Y);
+                    tmem_wait_ld16(X);
+                    tmem_wait_ld16(Y);
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+                        piece_max(X, mx);
+                        piece_max(Y, mx);
+                        const float mxc = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * c;
+                        float2 sum[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+                        piece_exp<0>(X, c, mxc, sum);
+                        tmem_st16(t0 + h * 128, X);
+                        if (h == 0) {
+                            mbar_wait(bar(kBarSFull + 2 * b + 1), ph, ab, prm.status);
+                            tc_fence_after();
+                            tmem_ld16(t0 + 128, X);
+                        }
+                        piece_exp<8>(Y, c, mxc, sum);
+                        tmem_st16(t0 + h * 128 + 16, Y);
+                        if (h == 0) tmem_ld16(t0 + 128 + 16, Y);
+                        const float2 s01 = __fadd2_rn(sum[0], sum[1]), s23 = __fadd2_rn(sum[2], sum[3]);
+                        tstat[(b * 8 + h * 4 + cq) * kTcRows + row] = make_float2(mxc, (s01.x + s01.y) + (s23.x + s23.y));
+                        if (h == 0) {
+                            tmem_wait_ld16(X);
+                            tmem_wait_ld16(Y);
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        mbar_wait(bar(kBarSFull + 2 * b + h), ph, ab, prm.status);
+                        tc_fence_after();
+                        tstat[(b * 8 + h * 4 + cq) * kTcRows + row] = pass1_chunk<false>(t0 + h * 128, h * 128 + cq * 32, nvalid, c);
+                    }
                 }
                 tmem_wait_st();
                 tc_fence_before();  // pass 2 reads these TMEM words from other lanes of the warp
