@@ -117,6 +117,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)   // never blocks
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
 __device__ __forceinline__ unsigned long long global_ns()
 {
     unsigned long long t;
@@ -549,14 +559,23 @@ cap_score_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                         float2 sum[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
                         piece_exp<0>(X, c, mxc, sum);
                         tmem_st16(t0 + h * 128, X);
-                        if (h == 0) {
-                            mbar_wait(bar(kBarSFull + 2 * b + 1), ph, ab, prm.status);
+                        // the second half's logits: fetched behind the next piece's exponentials if the tensor core has
+                        // delivered them by now (lane 0's answer for the whole warp: a phase that is complete stays complete)
+                        const bool early = h == 0 && __shfl_sync(0xffffffffu, mbar_test_wait(bar(kBarSFull + 2 * b + 1), ph) ? 1 : 0, 0);
+                        if (early) {
                             tc_fence_after();
                             tmem_ld16(t0 + 128, X);
                         }
                         piece_exp<8>(Y, c, mxc, sum);
                         tmem_st16(t0 + h * 128 + 16, Y);
-                        if (h == 0) tmem_ld16(t0 + 128 + 16, Y);
+                        if (h == 0) {
+                            if (!early) {
+                                mbar_wait(bar(kBarSFull + 2 * b + 1), ph, ab, prm.status);
+                                tc_fence_after();
+                                tmem_ld16(t0 + 128, X);
+                            }
+                            tmem_ld16(t0 + 128 + 16, Y);
+                        }
                         const float2 s01 = __fadd2_rn(sum[0], sum[1]), s23 = __fadd2_rn(sum[2], sum[3]);
                         tstat[(b * 8 + h * 4 + cq) * kTcRows + row] = make_float2(mxc, (s01.x + s01.y) + (s23.x + s23.y));
                         if (h == 0) {
