@@ -15,7 +15,9 @@
 //   pass 1   (16 epilogue warps; a thread owns one query row x two chunks of 32 columns,
 //            one in each half of the buffer) per chunk: maximum, e = 2^(x - max)
 //            written back over the logits, sum - one tensor-memory read and one
-//            write per logit; a quarter of the exponentials run on the FMA pipe;
+//            write per logit; a quarter of the exponentials run on the FMA pipe; the chunks move
+//            through two sets of 16 registers, the second chunk's first half being fetched behind the
+//            exponentials of the first chunk's second half;
 //   combine  (4 warps, one thread per query row) merges the eight (max, sum) pairs of
 //            its row into the slab's statistics and publishes them with one 8-byte
 //            store whose sum carries the launch's sign as a "fresh" mark; then reads
