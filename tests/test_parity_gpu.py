@@ -434,3 +434,28 @@ def test_seeded_random_configurations(seed):
         gpu = gpu_cycle(cfg, t, scorer, n=n)
         same, cnt = compare_cycle(cfg, t, gpu, n=n)
         assert cnt == cfg.units and same >= cnt - 1, (seed, scorer)
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_seeded_random_large_pots(seed):
+    """As above with pots of up to 20000 slots (the ranking kernels change their block shape at 4096, 8192 and 16384
+    slots), novelty scores quantised on a third of the cases so that ties straddle threads, and the chunk of a deferred
+    append starting anywhere on half of them."""
+    g = np.random.default_rng(77000 + seed)
+    dtype = "bf16" if g.random() < 0.7 else "f32"
+    d = int(g.choice([32, 64, 128]))
+    Hkv = int(g.choice([1, 2]))
+    G = int(g.choice([1, 2, 4]))
+    pot = int(g.choice([g.integers(70, 1400), g.integers(4000, 4200), g.integers(4097, 9000), g.integers(9000, 20000)]))
+    n = int(g.integers(max(2, pot // 2), pot + 1))
+    keep = int(g.integers(1, n))
+    T = int(g.integers(0, keep + 1))
+    cfg = inputs.small_config(cfg_id=3000 + seed, pot_size=pot, keep=keep, nuc_slots=T, cap_rows=int(g.integers(1, 12)),
+                              Hq=Hkv * G, Hkv=Hkv, d=d, dtype=dtype, layers=1, batch=int(g.integers(1, 3)))
+    t = inputs.make_cycle(cfg)
+    if g.random() < 0.3:
+        t["aux"] = np.round(t["aux"] * 8) / 8
+    deferred = int(g.integers(0, n)) if g.random() < 0.5 else None
+    gpu = gpu_cycle(cfg, t, ipot.IPOT_SCORER_AUTO, n=n, deferred_from=deferred)
+    same, cnt = compare_cycle(cfg, t, gpu, n=n)
+    assert cnt == cfg.units and same >= cnt - 1, seed
